@@ -215,3 +215,47 @@ def test_load_and_reputation_factors_shift_the_share():
     assert abs(n1 - Q / 3) < 5 * math.sqrt(Q * (1 / 3) * (2 / 3))   # weights 0.5 : 1
     W, sc, _ = o.window_weights(0, 0)
     assert W[1] * 2 == W[2] and sc[1] * 2 == sc[2]
+
+
+def test_tiny_weights_hit_interval_boundaries_exactly():
+    """Stakes of a few credits give weights of a few hundred, so draws land on interval
+    ends often; the pick must be the lane with prefix_excl <= r64 < prefix_incl."""
+    N, Q = 6, 6000
+    st, pa, rq = make_net(N, n_requests=Q, seed=77, flags=0, p_duel_ppm=0,
+                          peers=requester_first(N, credit0=np.array([10 ** 6, 1, 2, 3, 1, 2])))
+    o = Oracle(st, pa); o.bind_requests(rq)
+    o.dispatch_batch(0, Q)
+    res = o.results()
+    W, _, blk = o.window_weights(0, 0)
+    assert list(W[:6]) == [0, 256, 512, 768, 256, 512] and blk == 0
+    S = int(W.astype(object).sum()); incl = np.cumsum(W.astype(object))
+    on_edge = 0
+    for q in range(Q):
+        y = _philox(st.seed, q, 0, 0, ST_DRAW)
+        r64 = (((y[0] << 32) | y[1]) * S) >> 64
+        lane = next(c for c in range(32) if incl[c] > r64)
+        assert res["exec_a"][0, q] == lane
+        lo, hi = int(incl[lane]) - int(W[lane]), int(incl[lane])
+        assert (res["flags"][0, q] & 1) == int(r64 == lo or r64 == hi - 1)     # tolerance S // 100000 = 0
+        on_edge += int(r64 in [int(v) for v in incl[:6]] or r64 + 1 in [int(v) for v in incl[:6]])
+    assert on_edge > 20
+
+
+def test_truly_offline_peers_never_serve_or_judge():
+    """Peers that crashed but are still believed online get drawn, fail their probe,
+    and are skipped as judges."""
+    N, Q = 12, 5000
+    st, pa, rq = make_net(N, n_requests=Q, seed=41, flags=0, p_duel_ppm=1_000_000, n_judges=3, max_probes=6,
+                          peers=requester_first(N, credit0=10 ** 8))
+    o = Oracle(st, pa); o.bind_requests(rq)
+    dead = [2, 5, 6, 9]
+    for j in dead:
+        o.poke_peer(0, j, online=0)
+    o.dispatch_batch(0, Q); o.duel_judge()
+    res = o.results()
+    assert not np.isin(res["exec_a"][0], dead).any() and not np.isin(res["exec_b"][0], dead).any()
+    assert not np.isin(res["judges"][0], dead).any()
+    decided = np.isin(res["outcome"][0], (1, 2, 3))
+    assert decided.mean() > 0.9
+    assert np.all((res["judges"][0][decided] >= 0).sum(-1) == 3)     # 7 live candidates: always a full panel
+    assert o.stats_dict()["n_probes"] > 2 * Q                          # refused probes were spent on the dead

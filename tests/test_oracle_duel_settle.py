@@ -154,6 +154,9 @@ def test_credit_conserved_and_ledger_matches_results():
             dec = np.isin(res["outcome"][r], (1, 2))
             win = np.where(res["outcome"][r] == 1, res["exec_a"][r], res["exec_b"][r])[dec]
             assert np.array_equal(o.table("wins")[r], np.bincount(win, minlength=st.n_peers))
+            dl = np.isin(res["outcome"][r], (1, 2, 3))
+            both = np.concatenate([res["exec_a"][r][dl], res["exec_b"][r][dl]])
+            assert np.array_equal(o.table("duels")[r], np.bincount(both, minlength=st.n_peers))
 
 
 def test_pending_block_is_invisible_until_finalized():
@@ -177,6 +180,12 @@ def test_pending_block_is_invisible_until_finalized():
     assert np.array_equal(o2.table("credit") - pa2["credit0"], d)
     q = int(np.flatnonzero(res["outcome"][0] == 1)[0])
     assert (res["judges"][0, q] >= 0).sum() == 4
+    # queues: executors take the request's tokens, each judge reads both answers (len_in + 2 len_out)
+    bl = np.zeros(8, np.int64)
+    np.add.at(bl, res["exec_a"][0], 768); np.add.at(bl, res["exec_b"][0], 768)
+    np.add.at(bl, res["judges"][0].ravel(), 512 + 2 * 256)
+    assert np.array_equal(o2.table("backlog")[0], bl)
+    assert np.array_equal(o2.table("served")[0], np.bincount(np.concatenate([res["exec_a"][0], res["exec_b"][0]]), minlength=8))
 
 
 def test_lemma_1_mean_payoff_of_the_primary_executor():
@@ -257,6 +266,13 @@ def test_advance_time_and_latency_hand_cases():
     # deadline 2 * ceil(1000 * 1000 / 2000) = 1000 ms: only requests served by peer 2 (501 ms) meet it
     assert sd["slo_met"] == int((res[2:] == 2).sum())
     assert o.table("backlog")[0, 1] == 3000 + 1000 * (2 + int((res[2:] == 1).sum()))
+    # the drain runs at the effective (halved) rate while a priority window is active
+    st3, pa3, _ = make_net(2, peers={"prio_flag": 1}, p_prio_active_ppm=1_000_000)
+    o3 = Oracle(st3, pa3)
+    assert np.all(o3.table("cap_eff") == 1000)
+    o3.poke_peer(0, 0, backlog=5000)
+    o3.advance_time(1500)
+    assert o3.table("backlog")[0, 0] == 3500
     # priority window halves capacity while active
     st2, pa2, _ = make_net(400, peers={"prio_flag": 1}, p_prio_active_ppm=500_000, seed=3)
     o2 = Oracle(st2, pa2)
