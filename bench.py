@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the batched WWW.Serve network step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole path over one batch: advance -> gossip (on the steps its
+cadence selects) -> dispatch -> duel-and-judge -> settle.  Metric: simulated requests
+dispatched and settled per second.  One JSON line is printed by rank 0.
+
+Multi-GPU (`torchrun`, one process per GPU): replicas are independent, so every rank runs its
+own set of replicas (weak scaling, no data-path collective); timing is the max over ranks.
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "simulated requests dispatched+settled per second"
+UNIT = "requests/s"
+DEFAULT_WORKLOAD = "adversarial16k"          # the largest single-GPU configuration
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in out.strip().splitlines():
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def step_args(wl, s):
+    """(first, count, now_ms, gossip) of global step s; the request stream is reused cyclically
+    while simulated time keeps growing."""
+    n = wl.n_steps
+    cyc, k = divmod(s, n)
+    first = k * wl.batch
+    cnt = min(wl.batch, wl.n_requests - first)
+    t_end = int(wl.requests["t_ms"][0, -1]) + 1
+    return first, cnt, cyc * t_end + wl.step_now_ms(k), s % wl.gossip_every == 0
+
+
+def algorithmic_bytes(wl, stats_delta):
+    """Bytes the method must move (stated in the design notes):
+    gossip round: (k+2) * 8 * N^2 per replica (k+1 rows read, one written);
+    request path: 8 B record + 26 B result, plus a 256 B view window per request that offloads."""
+    st = wl.settings
+    gossip_round = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
+    offloaded = stats_delta["n_delegated"] + stats_delta["n_fallback_local"] + stats_delta["n_failed"]
+    req = stats_delta["n_requests"] * (8 + 26) + offloaded * 256
+    return gossip_round, req
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2603_20661_b200 import synth
+    from paper_2603_20661_b200.binding import Network, STAT_NAMES
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+
+    from paper_2603_20661_b200.sharding import max_over_ranks, replica_shard, sum_counters
+    wl0 = synth.make_workload(args.workload, seed=args.seed)
+    Rp = wl0.settings.n_replicas
+    # weak scaling: every rank runs the configuration's full replica count, on its own replica indices
+    off, _ = replica_shard(world * Rp, world, rank)
+    wl = synth.make_workload(args.workload, seed=args.seed, replica_offset=off)
+    st = wl.settings
+    net = Network(st, wl.peers, wl.batch, device=dev)
+    net.bind_requests(wl.requests, scores=False)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    reduce_max, reduce_sum_vec = max_over_ranks, sum_counters
+
+    W, K = args.warmup, args.steps
+    s = 0
+    for _ in range(W):
+        net.step(*step_args(wl, s)); s += 1
+    stats0 = net.stats()[-1].copy()
+    launches0 = net.kernel_launches()
+
+    # ---- timed region A: device-resident inputs --------------------------------------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    if sampler:
+        sampler.start()
+    ev0.record()
+    for _ in range(K):
+        net.step(*step_args(wl, s)); s += 1
+    ev1.record()
+    barrier()
+    ms = reduce_max(ev0.elapsed_time(ev1))
+    clocks = sampler.stop() if sampler else None
+    launches = net.kernel_launches() - launches0
+    stats1 = net.stats()[-1].copy()
+    delta = {k: int(b) - int(a) for k, a, b in zip(STAT_NAMES, stats0, stats1)}
+    total_requests = int(reduce_sum_vec(np.array([delta["n_requests"]], np.uint64))[0])
+    value = total_requests / (ms * 1e-3)
+
+    # ---- region B: same K steps with per-kernel events (roofline of the dominant kernel) ---
+    net.profile(True)
+    stats_b0 = net.stats()[-1].copy()
+    for _ in range(K):
+        net.step(*step_args(wl, s)); s += 1
+    prof = net.profile_read()
+    net.profile(False)
+    stats_b1 = net.stats()[-1].copy()
+    delta_b = {k: int(b) - int(a) for k, a, b in zip(STAT_NAMES, stats_b0, stats_b1)}
+    peak, peak_kind = measured_peaks()
+    g_bytes, req_bytes = algorithmic_bytes(wl, delta_b)
+    total_ms = sum(v[0] for v in prof.values())
+    dom = max(prof, key=lambda k: prof[k][0])
+    kernels = {k: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_ms} for k, v in prof.items()}
+
+    def roof(kernel, bytes_per_launch):
+        if kernel not in prof:
+            return None
+        t = prof[kernel][0] / prof[kernel][1] * 1e-3
+        ach = bytes_per_launch / t / 1e9
+        return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "peak_source": peak_kind, "traffic": None, "bytes_per_launch": bytes_per_launch,
+                "ms_per_launch": t * 1e3}
+
+    roof_merge = roof("k_gossip_merge", g_bytes)
+    roof_req = roof("k_step_fused", req_bytes / max(1, prof.get("k_step_fused", (0, 1))[1]))
+    roofline = roof_merge if dom == "k_gossip_merge" else roof_req
+
+    # ---- region C: end to end through host buffers ---------------------------------------------
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    Q = wl.n_requests
+    io = {"origin": pin(wl.requests["origin"].view(np.int32)), "len_in": pin(wl.requests["len_in"].view(np.int16)),
+          "len_out": pin(wl.requests["len_out"].view(np.int16)),
+          "exec_a": torch.empty((Rp, Q), dtype=torch.int32).pin_memory(),
+          "exec_b": torch.empty((Rp, Q), dtype=torch.int32).pin_memory(),
+          "judges": torch.empty((Rp, Q, 4), dtype=torch.int32).pin_memory(),
+          "outcome": torch.empty((Rp, Q), dtype=torch.uint8).pin_memory(),
+          "flags": torch.empty((Rp, Q), dtype=torch.uint8).pin_memory()}
+    for _ in range(min(W, 3)):
+        net.step_host(io, *step_args(wl, s)); s += 1
+    while s % wl.gossip_every:                 # start the timed steps on a gossip step, as region A did
+        net.step_host(io, *step_args(wl, s)); s += 1
+    stats_c0 = net.stats()[-1].copy()
+    barrier()
+    ev0.record()
+    for _ in range(K):
+        tot = net.step_host(io, *step_args(wl, s)); s += 1
+    ev1.record()
+    barrier()
+    ms_e2e = reduce_max(ev0.elapsed_time(ev1))
+    req_e2e = int(reduce_sum_vec(np.array([int(tot[0]) - int(stats_c0[0])], np.uint64))[0])
+    h2d = Rp * wl.batch * 8
+    d2h = Rp * wl.batch * 26 + 8 * len(STAT_NAMES)
+
+    line = None
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u64 views, i64 ledgers, fp32 scores", "data": "synthetic",
+            "config": {"workload": args.workload, "n_peers": st.n_peers, "n_replicas_per_gpu": Rp,
+                       "requests_per_step_per_gpu": Rp * wl.batch, "gossip_every": wl.gossip_every,
+                       "fanout_k": st.fanout_k, "entry": "wwws_step (fused dispatch+duel+settle)",
+                       "l2": "inputs larger than L2 (view buffers %.1f GB per GPU)" % (2 * 8 * st.n_peers ** 2 * Rp / 1e9)},
+            "clocks": clocks,
+            "e2e": {"value": req_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / K, "entry": "wwws_step_host, pinned host buffers"},
+            "gpu_launches": launches,
+            "roofline": roofline,
+            "roofline_request_path": roof_req,
+            "roofline_gossip_merge": roof_merge,
+            "kernels": kernels,
+            "step_mix": {k: delta[k] for k in ("n_requests", "n_delegated", "n_duel", "n_probes", "rounds")},
+        }
+    net.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return line
+
+
+def oracle_run(workload, seed, steps, warmup, replicas=1):
+    """Time the CPU oracle, as it stands, on `replicas` replicas of the workload: `warmup`
+    untimed steps, then `steps` timed ones.  Returns (requests/s, seconds, description)."""
+    from oracle import Oracle
+    from paper_2603_20661_b200 import synth
+    wl = synth.slice_replicas(synth.make_workload(workload, seed=seed), 0, replicas)
+    o = Oracle(wl.settings, wl.peers)
+    o.bind_requests(wl.requests)
+    s = 0
+    for _ in range(warmup):
+        f, c, now, g = step_args(wl, s); o.run_step(f, c, now, g); s += 1
+    n0 = o.stats_dict()["n_requests"]
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        f, c, now, g = step_args(wl, s); o.run_step(f, c, now, g); s += 1
+    dt = time.perf_counter() - t0
+    n = o.stats_dict()["n_requests"] - n0
+    rounds = sum(1 for k in range(warmup, warmup + steps) if k % wl.gossip_every == 0)
+    desc = (f"{replicas} replica(s) of {workload}, {steps} steps of {wl.batch} requests with {rounds} gossip round(s), "
+            f"single thread")
+    o.close()
+    return n / dt, dt, desc
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores (1 thread), bounded sample."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return None
+    from paper_2603_20661_b200 import synth
+    wl = synth.make_workload(args.workload, seed=args.seed, n_replicas=1, n_requests=1000)
+    K, W = args.steps, args.warmup
+    # keep the whole run to a few minutes: the oracle's gossip round costs O(k N^2) on one core
+    big = wl.settings.n_peers >= 8192
+    W_eff = min(W, wl.gossip_every) if big else W
+    K_eff = min(K, 2 * wl.gossip_every) if big else K
+    v, dt, desc = oracle_run(args.workload, args.seed, K_eff, W_eff, 1)
+    cb = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+    return {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": K_eff,
+            "warmup": W_eff, "ms_per_step": dt / K_eff * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u64 views, i64 ledgers, fp32 scores", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": desc}, "cpu_baseline": cb,
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        line = run_reference(args)
+        if line:
+            print(json.dumps(line))
+        return
+    line = run_gpu(args)
+    if line is not None:
+        if args.gpus == 1 and not args.no_cpu_baseline:
+            from paper_2603_20661_b200 import synth
+            ge = synth.make_workload(args.workload, n_replicas=1, n_requests=1000).gossip_every
+            v, dt, desc = oracle_run(args.workload, args.seed, ge, 0, 1)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
+                                    "seconds": dt}
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,200 @@
+// Per-peer kernels: initial state and views, time advance, queue fold, block finalization.
+#include "wwws_internal.cuh"
+
+namespace wwws {
+
+// Reputation-weighted stake in fp32: (float)stake * (float)(wins+1) / (float)(duels+2), each
+// operation rounded to nearest (no contraction), so the value equals the per-request formula.
+__device__ __forceinline__ float ledger_weight(const Net& n, int64_t stake, uint32_t wins, uint32_t duels)
+{
+    if (stake <= 0) return 0.0f;
+    const float sf = __ll2float_rn(stake);
+    float rep = 1.0f;
+    if (n.flags & 1u) rep = __fdiv_rn(__uint2float_rn(wins + 1u), __uint2float_rn(duels + 2u));
+    return __fmul_rn(sf, rep);
+}
+
+__global__ void k_peer_init(Net n, const int64_t* __restrict__ credit0, const uint8_t* __restrict__ online0,
+                            uint32_t init_stale_max)
+{
+    const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n.N) return;
+    const size_t x = size_t(r) * n.N + j;
+    n.online[x] = online0[x] ? 1 : 0;
+    n.ver[x] = init_stale_max + 1;
+    n.cap_eff[x] = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, 0);
+    n.backlog[x] = 0;
+    const int64_t c = credit0[x];
+    n.credit[x] = c;
+    const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
+    n.stake[x] = st;
+    n.wins[x] = 0; n.duels[x] = 0; n.served[x] = 0; n.served_local[x] = 0;
+    n.d_credit[x] = 0; n.d_wins[x] = 0; n.d_duels[x] = 0; n.d_backlog[x] = 0;
+    n.w_led[x] = ledger_weight(n, st, 0, 0);
+    n.self_entry[x] = 0;
+}
+
+// V[i][j] = entry of j at a version 0..init_stale_max old (own entry current).
+__global__ void k_view_init(Net n, uint32_t init_stale_max)
+{
+    const uint32_t r = blockIdx.z, i = blockIdx.y;
+    const uint32_t rg = r + n.replica_offset;
+    uint64_t* row = n.view + (size_t(r) * n.N + i) * n.ld;
+    for (uint32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < n.ld; j += gridDim.x * blockDim.x) {
+        uint64_t e = 0;
+        if (j < n.N) {
+            const size_t x = size_t(r) * n.N + j;
+            uint32_t stale = 0;
+            if (init_stale_max != 0 && i != j) stale = below(draw(n, i, j, rg, kInit).w[0], init_stale_max + 1);
+            e = pack_entry(n.ver[x] - stale, n.online[x] == 0, uint64_t(n.cap_eff[x]) * n.misreport[x], 0);
+        }
+        row[j] = e;
+    }
+}
+
+__global__ void k_advance(Net n, uint32_t dt_ms, uint32_t now_ms)
+{
+    const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n.N) return;
+    const size_t x = size_t(r) * n.N + j;
+    const uint32_t cap = n.cap_eff[x];
+    if (n.online[x]) {
+        const int64_t done = int64_t(uint64_t(cap) * dt_ms / 1000u);
+        const int64_t b = n.backlog[x];
+        n.backlog[x] = b > done ? b - done : 0;
+    }
+    n.cap_eff[x] = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, now_ms);
+}
+
+// End of a settlement: queues take the batch's work; with `finalize` the pending block is
+// folded into the ledger, stakes and derived weights are refreshed and credit is summed.
+__global__ void k_fold(Net n, int finalize)
+{
+    const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    long long csum = 0;
+    if (j < n.N) {
+        const size_t x = size_t(r) * n.N + j;
+        const long long db = n.d_backlog[x];
+        if (db) { n.backlog[x] += db; n.d_backlog[x] = 0; }
+        if (finalize) {
+            const int64_t c = n.credit[x] + n.d_credit[x];
+            const uint32_t w = n.wins[x] + n.d_wins[x], d = n.duels[x] + n.d_duels[x];
+            n.credit[x] = c; n.wins[x] = w; n.duels[x] = d;
+            n.d_credit[x] = 0; n.d_wins[x] = 0; n.d_duels[x] = 0;
+            const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
+            n.stake[x] = st;
+            n.w_led[x] = ledger_weight(n, st, w, d);
+            csum = c;
+        }
+    }
+    if (finalize) {
+        for (int o = 16; o; o >>= 1) csum += __shfl_down_sync(0xffffffffu, csum, o);
+        if ((threadIdx.x & 31) == 0 && csum) atomicAdd((unsigned long long*)&n.credit_check[r], (unsigned long long)csum);
+    }
+}
+
+__global__ void k_finalize_check(Net n)
+{
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n.Rp) return;
+    if (n.credit_check[r] != n.credit_total0[r]) set_error(n, eInvariant, r);
+    n.credit_check[r] = 0;
+    n.stats[size_t(r) * sCount + sBlocks] += 1;
+}
+
+// Re-derive stake and weight from the ledger as it stands (after a table import).
+__global__ void k_rederive(Net n)
+{
+    const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n.N) return;
+    const size_t x = size_t(r) * n.N + j;
+    const int64_t c = n.credit[x];
+    const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
+    n.stake[x] = st;
+    n.w_led[x] = ledger_weight(n, st, n.wins[x], n.duels[x]);
+}
+
+// credit_total per replica = sum of finalized and pending credit.
+__global__ void k_credit_total(Net n)
+{
+    const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    long long s = 0;
+    if (j < n.N) { const size_t x = size_t(r) * n.N + j; s = n.credit[x] + n.d_credit[x]; }
+    for (int o = 16; o; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+    if ((threadIdx.x & 31) == 0 && s) atomicAdd(&n.stats[size_t(r) * sCount + sCreditTotal], (unsigned long long)s);
+}
+
+__global__ void k_zero_credit_total(Net n)
+{
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < n.Rp) n.stats[size_t(r) * sCount + sCreditTotal] = 0;
+}
+
+static dim3 peer_grid(const Net& n) { return dim3((n.N + 255) / 256, n.Rp); }
+
+void launch_peer_init(const Net& n, const int64_t* credit0, const uint8_t* online0, uint32_t init_stale_max, const LaunchCtx& c)
+{
+    { Timed t(c, kPeerInit); k_peer_init<<<peer_grid(n), 256, 0, c.stream>>>(n, credit0, online0, init_stale_max); }
+    const uint32_t bx = (n.ld + 255) / 256 > 64 ? 64 : (n.ld + 255) / 256;
+    // grid.y / grid.z limits (65535): rows go in y, replicas in z
+    { Timed t(c, kViewInit); k_view_init<<<dim3(bx, n.N, n.Rp), 256, 0, c.stream>>>(n, init_stale_max); }
+}
+
+void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c)
+{
+    Timed t(c, kAdvance);
+    k_advance<<<peer_grid(n), 256, 0, c.stream>>>(n, dt_ms, now_ms);
+}
+
+void launch_fold(const Net& n, int finalize, const LaunchCtx& c)
+{
+    { Timed t(c, kFold); k_fold<<<peer_grid(n), 256, 0, c.stream>>>(n, finalize); }
+    if (finalize) { Timed t(c, kFinalizeCheck); k_finalize_check<<<(n.Rp + 127) / 128, 128, 0, c.stream>>>(n); }
+}
+
+void launch_rederive(const Net& n, const LaunchCtx& c)
+{
+    Timed t(c, kRederive);
+    k_rederive<<<peer_grid(n), 256, 0, c.stream>>>(n);
+}
+
+void launch_credit_total(const Net& n, const LaunchCtx& c)
+{
+    { Timed t(c, kCreditTotal); k_zero_credit_total<<<(n.Rp + 127) / 128, 128, 0, c.stream>>>(n); }
+    { Timed t(c, kCreditTotal); k_credit_total<<<peer_grid(n), 256, 0, c.stream>>>(n); }
+}
+
+// ---- optional per-kernel event timing ------------------------------------------------------------
+
+void Profiler::begin(int id, cudaStream_t s)
+{
+    Pair p;
+    if (!pool.empty()) { p = pool.back(); pool.pop_back(); }
+    else { cudaEventCreate(&p.a); cudaEventCreate(&p.b); }
+    p.id = id;
+    cudaEventRecord(p.a, s);
+    used.push_back(p);
+}
+void Profiler::end(cudaStream_t s) { cudaEventRecord(used.back().b, s); }
+void Profiler::collect()
+{
+    for (Pair& p : used) {
+        cudaEventSynchronize(p.b);
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, p.a, p.b) == cudaSuccess) { ms[p.id] += t; count[p.id] += 1; }
+        pool.push_back(p);
+    }
+    used.clear();
+}
+void Profiler::reset()
+{
+    collect();
+    for (int k = 0; k < kKernelCount; ++k) { ms[k] = 0; count[k] = 0; }
+}
+Profiler::~Profiler()
+{
+    for (Pair& p : used) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+    for (Pair& p : pool) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+}
+
+}  // namespace wwws

@@ -1,0 +1,118 @@
+// Device-side state layout and small helpers shared by the wwws kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace wwws {
+
+constexpr uint32_t kWin = 32;                 // candidate window = one warp
+constexpr uint64_t kOffBit = 1ull << 39;
+constexpr uint32_t kCapMax = (1u << 19) - 1;
+constexpr uint32_t kQMax = (1u << 20) - 1;
+
+// Random stages: the fourth counter word is stage + 256 * attempt.
+enum : uint32_t { kOrigin = 1, kDraw = 2, kProbe = 3, kJudge = 4, kGossip = 5, kChurn = 6, kPrio = 7, kInit = 8 };
+
+// Per-replica counters, in the order of wwws_stats_t.
+enum : uint32_t { sRequests, sLocal, sFallback, sDropped, sFailed, sDelegated, sDuel, sDuelCancelled, sDraw,
+                  sJudgeEvals, sProbes, sNear, sSloMet, sSumLat, sOfflineMarks, sRounds, sBlocks, sCreditTotal, sCount };
+
+// Device error word codes (subset of wwws_status).
+enum : uint32_t { eArg = 1, eRange = 4, eInvariant = 6 };
+
+// Everything a kernel needs, passed by value.  Per-peer arrays are [Rp][N]; the view is
+// [Rp][N][ld] with ld = N rounded up to 32 so that a candidate window is one aligned
+// 256-byte segment; padding columns stay 0 ("never heard of").
+struct Net {
+    uint32_t N, Rp, ld, n_blk, replica_offset;
+    uint32_t key0, key1;
+    uint32_t fanout_k, gossip_tries, max_probes, n_judges;
+    uint32_t p_duel, p_noise, p_leave, p_join, p_prio;
+    uint32_t prio_window_ms, util_window_ms, cap_ref, slo_num, slo_den, hop_ms, flags, n_rank;
+    int64_t R, R_add, P;
+    float uwf;                                   // util_window_ms / 1000 in fp32
+    // view double buffer
+    uint64_t* view; uint64_t* view_new;
+    // hidden / policy (constant after creation)
+    const uint32_t* cap_true; const uint32_t* quality; const uint16_t* stake_pm; const uint16_t* offload_util_pm;
+    const uint16_t* accept_util_pm; const uint32_t* offload_ppm; const uint32_t* accept_ppm;
+    const uint8_t* misreport; const uint8_t* prio_flag;
+    // dynamic
+    uint8_t* online; uint32_t* cap_eff; int64_t* backlog; uint32_t* ver;
+    // ledger
+    int64_t* credit; int64_t* stake; uint32_t* wins; uint32_t* duels;
+    unsigned long long* served; unsigned long long* served_local;
+    // pending block and pending queue growth
+    long long* d_credit; uint32_t* d_wins; uint32_t* d_duels; long long* d_backlog;
+    // derived: (float)stake * smoothed win rate, refreshed whenever the ledger is finalized
+    float* w_led;
+    // gossip scratch: this round's self entries and chosen partners
+    uint64_t* self_entry; int32_t* partner;     // partner is [Rp][N][4]
+    // dispatch -> duel continuation, [Rp][max_batch]
+    uint2* cont; uint32_t max_batch;
+    const uint32_t* rank_cdf;
+    unsigned long long* stats;                   // [Rp][sCount]
+    const int64_t* credit_total0; long long* credit_check;   // [Rp]
+    uint32_t* err;                               // [2]: code, detail
+    // bound requests / results
+    const uint32_t* origin; const uint16_t* len_in; const uint16_t* len_out; uint64_t Q;
+    int32_t* exec_a; int32_t* exec_b; int32_t* judges; uint8_t* outcome; uint8_t* rflags;
+    float* score_a; float* score_sum;
+};
+
+struct Rnd4 { uint32_t w[4]; };
+
+// Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11).
+__device__ __forceinline__ Rnd4 philox(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3)
+{
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    Rnd4 r; r.w[0] = c0; r.w[1] = c1; r.w[2] = c2; r.w[3] = c3;
+    return r;
+}
+
+__device__ __forceinline__ Rnd4 draw(const Net& n, uint32_t index, uint32_t slot, uint32_t rg, uint32_t stage)
+{
+    return philox(n.key0, n.key1, index, slot, rg, stage);
+}
+
+__device__ __forceinline__ uint32_t ppm(uint32_t x) { return __umulhi(x, 1000000u); }
+__device__ __forceinline__ uint32_t below(uint32_t x, uint32_t m) { return __umulhi(x, m); }
+
+__device__ __forceinline__ uint64_t pack_entry(uint32_t ver, bool offline, uint64_t cap, uint64_t q)
+{
+    cap = cap > kCapMax ? kCapMax : cap;
+    q = q > kQMax ? kQMax : q;
+    return (uint64_t(ver) << 40) | (offline ? kOffBit : 0ull) | (cap << 20) | q;
+}
+
+// floor(min(1000, backlog*1000/denom)) >= thr  without the division.
+__device__ __forceinline__ bool util_at_least(uint32_t cap_eff, int64_t backlog, uint32_t util_window_ms, uint32_t thr)
+{
+    if (thr == 0) return true;
+    if (thr > 1000) return false;
+    if (cap_eff == 0) return true;
+    uint64_t denom = uint64_t(cap_eff) * util_window_ms / 1000u;
+    if (denom < 1) denom = 1;
+    return uint64_t(backlog) * 1000ull >= uint64_t(thr) * denom;
+}
+
+__device__ __forceinline__ uint32_t cap_eff_at(const Net& n, uint32_t cap_true, bool prio, uint32_t j, uint32_t rg,
+                                               uint32_t now_ms)
+{
+    if (!prio) return cap_true;
+    const uint32_t w = now_ms / n.prio_window_ms;
+    return ppm(draw(n, j, w, rg, kPrio).w[0]) < n.p_prio ? cap_true / 2 : cap_true;
+}
+
+__device__ __forceinline__ void set_error(const Net& n, uint32_t code, uint32_t detail)
+{
+    if (atomicCAS(&n.err[0], 0u, code) == 0u) n.err[1] = detail;
+}
+
+}  // namespace wwws

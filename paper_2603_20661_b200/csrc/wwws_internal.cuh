@@ -1,0 +1,52 @@
+// Launchers of the wwws kernels (internal to the library) and the optional per-kernel timer.
+#pragma once
+#include <vector>
+
+#include "wwws_device.cuh"
+
+namespace wwws {
+
+// Kernel classes, for launch counts and optional event timing.
+enum KernelId : int { kPeerInit, kViewInit, kAdvance, kFold, kFinalizeCheck, kRederive, kCreditTotal, kGossipPeer,
+                      kGossipMerge, kGossipFixup, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
+
+// When enabled, every launch is bracketed by two events on the launching stream; read()
+// synchronises and returns the summed device time per kernel class.
+struct Profiler {
+    bool enabled = false;
+    struct Pair { cudaEvent_t a, b; int id; };
+    std::vector<Pair> used;
+    std::vector<Pair> pool;
+    double ms[kKernelCount] = {};
+    uint64_t count[kKernelCount] = {};
+    void begin(int id, cudaStream_t s);
+    void end(cudaStream_t s);
+    void collect();              // synchronises the events recorded so far
+    void reset();
+    ~Profiler();
+};
+
+struct LaunchCtx {
+    cudaStream_t stream;
+    uint64_t* launches;          // total kernels launched
+    Profiler* prof;
+};
+
+struct Timed {                   // RAII bracket around one launch
+    const LaunchCtx& c;
+    Timed(const LaunchCtx& ctx, int id) : c(ctx) { *c.launches += 1; if (c.prof && c.prof->enabled) c.prof->begin(id, c.stream); }
+    ~Timed() { if (c.prof && c.prof->enabled) c.prof->end(c.stream); }
+};
+
+void launch_peer_init(const Net& n, const int64_t* credit0, const uint8_t* online0, uint32_t init_stale_max, const LaunchCtx& c);
+void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c);
+void launch_fold(const Net& n, int finalize, const LaunchCtx& c);
+void launch_rederive(const Net& n, const LaunchCtx& c);
+void launch_credit_total(const Net& n, const LaunchCtx& c);
+void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c);
+void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
+void launch_duel(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
+void launch_settle(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
+void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
+
+}  // namespace wwws

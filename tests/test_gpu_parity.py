@@ -1,0 +1,170 @@
+"""GPU parity: the CUDA library against the CPU oracle, bit for bit, through the C-ABI.
+
+Views, ledgers, queues, executor choices, duel pairings, judge panels, outcomes and
+counters must be identical; fp32 scores within 1e-5 relative.
+"""
+import numpy as np
+import pytest
+
+from oracle import Oracle
+from paper_2603_20661_b200 import synth
+from tests.helpers import assert_same_state, make_net, requester_first
+
+pytestmark = pytest.mark.gpu
+
+
+def _pair(wl, max_batch=None):
+    from paper_2603_20661_b200.binding import Network
+    g = Network(wl.settings, wl.peers, max_batch or wl.batch)
+    g.bind_requests(wl.requests)
+    o = Oracle(wl.settings, wl.peers)
+    o.bind_requests(wl.requests)
+    return g, o
+
+
+CASES = [
+    ("tiny", {}, None),
+    ("tiers64", dict(n_requests=6000), None),
+    ("zipf1k", dict(n_replicas=3, n_requests=2500), None),
+    ("churn4k", dict(n_replicas=2, n_requests=6000, n_peers=1100), None),      # ragged last block (1100 = 34*32+12)
+    ("adversarial16k", dict(n_replicas=2, n_requests=3000, n_peers=2048), None),
+]
+
+
+@pytest.mark.parametrize("name,kw,steps", CASES, ids=[c[0] for c in CASES])
+def test_six_calls_match_oracle_after_every_call(name, kw, steps):
+    wl = synth.make_workload(name, **kw)
+    g, o = _pair(wl)
+    n = wl.n_steps if steps is None else steps
+    assert_same_state(g, o, "after create")
+    for s in range(n):
+        first = s * wl.batch
+        cnt = min(wl.batch, wl.n_requests - first)
+        gossip = s % wl.gossip_every == 0
+        full = s < 3 or s == n - 1          # compare after every call early on, then once per step
+        for sim in (g, o):
+            sim.advance_time(wl.step_now_ms(s))
+        if full:
+            assert_same_state(g, o, f"step {s} advance", views=False)
+        if gossip:
+            g.gossip_round(); o.gossip_round()
+            if full or s % 7 == 0:
+                assert_same_state(g, o, f"step {s} gossip")
+        g.dispatch_batch(first, cnt); o.dispatch_batch(first, cnt)
+        if full:
+            assert_same_state(g, o, f"step {s} dispatch", upto=first + cnt, views=False, stats=False)
+        g.duel_judge(); o.duel_judge()
+        if full:
+            assert_same_state(g, o, f"step {s} duel", upto=first + cnt, views=False, stats=False)
+        g.settle_credits(True); o.settle_credits(True)
+        assert_same_state(g, o, f"step {s} settle", upto=first + cnt, views=False)
+    assert_same_state(g, o, "end", upto=wl.n_requests)
+    assert o.error() == 0
+    sd = g.stats_dict()
+    assert sd["n_requests"] == wl.settings.n_replicas * wl.n_requests
+    assert sd["credit_total"] == int(wl.peers["credit0"].sum())
+
+
+@pytest.mark.parametrize("name,kw,steps", CASES, ids=[c[0] for c in CASES])
+def test_fused_step_matches_oracle(name, kw, steps):
+    wl = synth.make_workload(name, **kw)
+    g, o = _pair(wl)
+    for s in range(wl.n_steps):
+        first = s * wl.batch
+        cnt = min(wl.batch, wl.n_requests - first)
+        gossip = s % wl.gossip_every == 0
+        fin = s % 3 != 1                     # leave some blocks pending across steps
+        g.step(first, cnt, wl.step_now_ms(s), gossip, fin)
+        o.run_step(first, cnt, wl.step_now_ms(s), gossip, fin)
+        if s < 2 or s % 5 == 0:
+            assert_same_state(g, o, f"fused step {s}", upto=first + cnt, views=gossip)
+    assert_same_state(g, o, "fused end", upto=wl.n_requests)
+
+
+def test_step_host_roundtrip_matches_oracle():
+    import torch
+    from paper_2603_20661_b200.binding import Network
+    wl = synth.make_workload("zipf1k", n_replicas=2, n_requests=1500, n_peers=256)
+    o = Oracle(wl.settings, wl.peers); o.bind_requests(wl.requests)
+    g = Network(wl.settings, wl.peers, wl.batch)
+    Rp, Q = wl.settings.n_replicas, wl.n_requests
+    # device arrays start as garbage: everything must arrive through the host copies
+    g.bind_requests({k: np.full((Rp, Q), 7, v.dtype) for k, v in wl.requests.items()}, scores=False)
+    pin = lambda a: torch.from_numpy(a.copy()).pin_memory()
+    io = {"origin": pin(wl.requests["origin"].view(np.int32)), "len_in": pin(wl.requests["len_in"].view(np.int16)),
+          "len_out": pin(wl.requests["len_out"].view(np.int16)),
+          "exec_a": torch.full((Rp, Q), -9, dtype=torch.int32).pin_memory(),
+          "exec_b": torch.full((Rp, Q), -9, dtype=torch.int32).pin_memory(),
+          "judges": torch.full((Rp, Q, 4), -9, dtype=torch.int32).pin_memory(),
+          "outcome": torch.zeros((Rp, Q), dtype=torch.uint8).pin_memory(),
+          "flags": torch.zeros((Rp, Q), dtype=torch.uint8).pin_memory()}
+    for s in range(wl.n_steps):
+        first = s * wl.batch
+        tot = g.step_host(io, first, wl.batch, wl.step_now_ms(s), s % wl.gossip_every == 0)
+        o.run_step(first, wl.batch, wl.step_now_ms(s), s % wl.gossip_every == 0)
+        assert np.array_equal(tot, o.stats()[-1])
+    ro = o.results()
+    for k in ("exec_a", "exec_b", "judges", "outcome", "flags"):
+        assert np.array_equal(io[k].numpy(), ro[k]), k
+    assert_same_state(g, o, "host path end", upto=Q)
+
+
+def test_determinism_and_replica_sharding():
+    """Same seed twice gives the same bytes; replicas [2,4) run alone (replica_offset = 2)
+    give the same results as inside the 4-replica network."""
+    from paper_2603_20661_b200.binding import Network
+    wl = synth.make_workload("churn4k", n_replicas=4, n_requests=3000, n_peers=512)
+    outs = []
+    for _ in range(2):
+        g = Network(wl.settings, wl.peers, wl.batch); g.bind_requests(wl.requests)
+        for s in range(wl.n_steps):
+            g.step(s * wl.batch, wl.batch, wl.step_now_ms(s), s % wl.gossip_every == 0)
+        outs.append((g.results(), g.view(), g.table("credit"), g.stats()))
+        g.close()
+    for k in outs[0][0]:
+        assert np.array_equal(outs[0][0][k], outs[1][0][k])
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][3], outs[1][3])
+    half = synth.slice_replicas(wl, 2, 4)
+    g = Network(half.settings, half.peers, half.batch); g.bind_requests(half.requests)
+    for s in range(half.n_steps):
+        g.step(s * half.batch, half.batch, half.step_now_ms(s), s % half.gossip_every == 0)
+    res = g.results()
+    for k in res:
+        assert np.array_equal(res[k], outs[0][0][k][2:4])
+    assert np.array_equal(g.view(), outs[0][1][2:4]) and np.array_equal(g.table("credit"), outs[0][2][2:4])
+    assert np.array_equal(g.stats()[:2], outs[0][3][2:4])
+
+
+def test_edge_cases_match_oracle():
+    """Degenerate networks: two peers, a single request, everybody offline, nobody willing,
+    requester-only origin, ragged window, duel probability one with tiny candidate sets."""
+    from paper_2603_20661_b200.binding import Network
+    rng = np.random.default_rng(5)
+    cases = []
+    cases.append(make_net(2, n_requests=64, seed=1, p_duel_ppm=1_000_000))                       # never a challenger
+    cases.append(make_net(3, n_requests=64, seed=2, p_duel_ppm=1_000_000, n_judges=4))          # never a judge
+    cases.append(make_net(4, n_requests=1, seed=3))
+    cases.append(make_net(33, n_requests=200, seed=4, origin=rng.integers(0, 33, 200), p_duel_ppm=500_000))
+    cases.append(make_net(40, n_requests=200, seed=5, origin=rng.integers(0, 40, 200),
+                          peers={"online0": np.zeros(40, np.uint8)}))                            # all dropped
+    cases.append(make_net(40, n_requests=200, seed=6, origin=rng.integers(0, 40, 200),
+                          peers={"accept_ppm": 0}))                                              # all fallback
+    cases.append(make_net(12, n_requests=300, seed=7, p_duel_ppm=1_000_000, n_judges=2, max_probes=2,
+                          peers=requester_first(12, accept_ppm=500_000, credit0=10 ** 7)))       # failed (-4)
+    cases.append(make_net(64, n_requests=300, seed=8, origin=rng.integers(0, 64, 300), p_duel_ppm=300_000,
+                          p_noise_ppm=500_000, hop_ms=25, flags=0, p_leave_ppm=200_000, p_join_ppm=500_000,
+                          peers={"stake_pm": rng.integers(0, 1001, 64), "credit0": rng.integers(0, 300, 64),
+                                 "prio_flag": 1, "misreport_mul": rng.integers(1, 5, 64)}))
+    for ci, (st, pa, rq) in enumerate(cases):
+        g = Network(st, pa, 128); g.bind_requests(rq)
+        o = Oracle(st, pa); o.bind_requests(rq)
+        Q = rq["origin"].shape[1]
+        first = 0
+        step = 0
+        while first < Q:
+            cnt = min(100, Q - first)
+            for sim in (g, o):
+                sim.run_step(first, cnt, 700 * (step + 1), True, step % 2 == 0)
+            assert_same_state(g, o, f"edge case {ci} step {step}", upto=first + cnt)
+            first += cnt; step += 1
+        g.close()
