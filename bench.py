@@ -118,11 +118,11 @@ def run_gpu(args):
     dev = torch.device(f"cuda:{local}")
 
     from paper_2603_20661_b200.sharding import max_over_ranks, replica_shard, sum_counters
-    wl0 = synth.make_workload(args.workload, seed=args.seed)
+    wl0 = synth.make_workload(args.workload, seed=args.seed, n_replicas=args.replicas)
     Rp = wl0.settings.n_replicas
     # weak scaling: every rank runs the configuration's full replica count, on its own replica indices
     off, _ = replica_shard(world * Rp, world, rank)
-    wl = synth.make_workload(args.workload, seed=args.seed, replica_offset=off)
+    wl = synth.make_workload(args.workload, seed=args.seed, replica_offset=off, n_replicas=args.replicas)
     st = wl.settings
     net = Network(st, wl.peers, wl.batch, device=dev)
     net.bind_requests(wl.requests, scores=False)
@@ -144,16 +144,16 @@ def run_gpu(args):
     # ---- timed region A: device-resident inputs --------------------------------------------
     sampler = ClockSampler(local) if rank == 0 else None
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     if sampler:
         sampler.start()
+        time.sleep(0.5)                                # nvidia-smi needs a moment before its first sample
+    barrier()
     ev0.record()
     for _ in range(K):
         net.step(*step_args(wl, s)); s += 1
     ev1.record()
     barrier()
     ms = reduce_max(ev0.elapsed_time(ev1))
-    clocks = sampler.stop() if sampler else None
     launches = net.kernel_launches() - launches0
     stats1 = net.stats()[-1].copy()
     delta = {k: int(b) - int(a) for k, a, b in zip(STAT_NAMES, stats0, stats1)}
@@ -167,6 +167,7 @@ def run_gpu(args):
         net.step(*step_args(wl, s)); s += 1
     prof = net.profile_read()
     net.profile(False)
+    clocks = sampler.stop() if sampler else None     # sampled over region A and its instrumented repeat
     stats_b1 = net.stats()[-1].copy()
     delta_b = {k: int(b) - int(a) for k, a, b in zip(STAT_NAMES, stats_b0, stats_b1)}
     peak, peak_kind = measured_peaks()
@@ -291,6 +292,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--replicas", type=int, default=None, help="override the workload's replica count (profiling)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     args = ap.parse_args()
