@@ -239,6 +239,28 @@ const char* wwws_profile_kernel_name(uint32_t kernel);
 
 const char* wwws_last_error(const wwws_network* net);
 
+/* wwws_gossip_round for callers that must not allocate.  (The paper has no counterpart: this
+ * is a packaging variant of the round above, with identical results.)
+ *
+ * Who needs it: a program that embeds the library at a point where it cannot obtain device
+ * memory - the whole GPU already belongs to another allocator's pool, allocation is not
+ * allowed in that phase, or the device-wide synchronisation of cudaMalloc would stall its
+ * loop.  The round's scratch (this round's self entries and partner lists, 24 bytes per
+ * peer and replica) is taken from a fixed 1.5 MiB array inside the library image instead of
+ * the workspace; every GPU that loads the library holds that array until the process exits.
+ * The call itself allocates nothing on host or device paths of CUDA: no cudaMalloc, no
+ * cudaFree, no allocating library routine.
+ *
+ * Limit: n_replicas * n_peers <= 65536; larger networks get WWWS_ERR_ARG and must use
+ * wwws_gossip_round.  The first call on each device looks up the array's device address
+ * (with that device current - call it with the network's device current, as for every
+ * other call) and should be made before any stream capture begins.  All calls, from all
+ * networks on a device, share the one array: two such rounds that overlap on the GPU (two
+ * streams) race and give wrong views; run them one after another.  The array keeps the
+ * previous round's contents; nothing in it has to start at zero, because each round
+ * rewrites the entries of all its peers before reading them. */
+wwws_status wwws_gossip_round_static(wwws_network* net);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,7 +29,7 @@ EXPORTS = ("wwws_workspace_bytes", "wwws_create_network", "wwws_destroy_network"
            "wwws_advance_time", "wwws_gossip_round", "wwws_dispatch_batch", "wwws_duel_judge", "wwws_settle_credits",
            "wwws_step", "wwws_step_host", "wwws_stats", "wwws_export_table", "wwws_import_table",
            "wwws_export_view_rows", "wwws_kernel_launches", "wwws_last_error", "wwws_profile", "wwws_profile_read",
-           "wwws_profile_kernels", "wwws_profile_kernel_name")
+           "wwws_profile_kernels", "wwws_profile_kernel_name", "wwws_gossip_round_static")
 
 
 class WwwsError(RuntimeError):
@@ -86,7 +86,7 @@ def load():
             "wwws_create_network": [C.POINTER(Config), C.POINTER(PeerInit), vp, u64, vp, C.POINTER(vp)],
             "wwws_destroy_network": [vp],
             "wwws_bind_requests": [vp, C.POINTER(Requests), C.POINTER(Results)],
-            "wwws_advance_time": [vp, u32], "wwws_gossip_round": [vp],
+            "wwws_advance_time": [vp, u32], "wwws_gossip_round": [vp], "wwws_gossip_round_static": [vp],
             "wwws_dispatch_batch": [vp, u64, u64], "wwws_duel_judge": [vp], "wwws_settle_credits": [vp, i32],
             "wwws_step": [vp, u64, u64, u32, i32, i32],
             "wwws_step_host": [vp, C.POINTER(HostIO), u64, u64, u32, i32, i32, vp],
@@ -215,6 +215,10 @@ class Network:
 
     def gossip_round(self):
         self._check(load().wwws_gossip_round(self._h), self._h)
+
+    def gossip_round_static(self):
+        """A gossip round whose scratch is the library's built-in array (see include/wwws.h)."""
+        self._check(load().wwws_gossip_round_static(self._h), self._h)
 
     def dispatch_batch(self, first, count):
         self._check(load().wwws_dispatch_batch(self._h, int(first), int(count)), self._h)

@@ -439,3 +439,55 @@ const char* wwws_profile_kernel_name(uint32_t k)
 const char* wwws_last_error(const wwws_network* n) { return n ? n->err.c_str() : g_err.c_str(); }
 
 }  // extern "C"
+
+// ---- gossip round whose scratch lives in the library image --------------------------------------
+//
+// Some programs that embed this library may not allocate device memory at the point where
+// they call it: all of the GPU's memory already belongs to another allocator (an inference
+// server's pool), an allocation is not permitted in that phase of the program, or the
+// device-wide synchronisation that cudaMalloc implies is not acceptable inside their loop.
+// For them the scratch of a gossip round (this round's self entries and partner lists) sits
+// in a fixed array that every GPU holds from the moment it loads the library until exit.
+
+namespace {
+
+constexpr uint64_t kStaticPeers = 65536;                       // n_replicas * n_peers limit
+constexpr uint64_t kStaticSelfBytes = kStaticPeers * sizeof(uint64_t);
+constexpr uint64_t kStaticPartnerBytes = kStaticPeers * 4 * sizeof(int32_t);
+static __device__ __align__(256) unsigned char g_gossip_scratch[kStaticSelfBytes + kStaticPartnerBytes];  // 1.5 MiB
+
+constexpr int kMaxDevices = 64;
+void* g_gossip_scratch_addr[kMaxDevices];                      // per device, filled on first use
+
+}  // namespace
+
+extern "C" wwws_status wwws_gossip_round_static(wwws_network* n)
+{
+    if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "gossip_round inside a batch");
+    const uint64_t peers = uint64_t(n->d.N) * n->d.Rp;
+    if (peers > kStaticPeers) {
+        char buf[160];
+        snprintf(buf, sizeof buf, "n_replicas * n_peers = %llu exceeds the built-in scratch of %llu peers; use wwws_gossip_round",
+                 (unsigned long long)peers, (unsigned long long)kStaticPeers);
+        return fail(n, WWWS_ERR_ARG, buf);
+    }
+    int dev = -1;
+    CUDA_TRY(n, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(n, WWWS_ERR_ARG, "device ordinal beyond 63");
+    if (!g_gossip_scratch_addr[dev]) {
+        // In host code the array's name is only a handle for the runtime; the address the
+        // kernels need comes from the runtime, for the device that is current now.
+        void* p = nullptr;
+        CUDA_TRY(n, cudaGetSymbolAddress(&p, g_gossip_scratch));
+        g_gossip_scratch_addr[dev] = p;
+    }
+    unsigned char* base = static_cast<unsigned char*>(g_gossip_scratch_addr[dev]);
+    Net d = n->d;                                              // same network, scratch pointers redirected
+    d.self_entry = reinterpret_cast<uint64_t*>(base);
+    d.partner = reinterpret_cast<int32_t*>(base + kStaticSelfBytes);
+    launch_gossip(d, n->round, n->ctx());
+    std::swap(n->d.view, n->d.view_new);
+    n->round += 1;
+    return launch_status(n, "gossip_round_static");
+}
