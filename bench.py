@@ -94,10 +94,11 @@ def step_args(wl, s):
 
 def algorithmic_bytes(wl, stats_delta):
     """Bytes the method must move (stated in the design notes):
-    gossip round: (k+2) * 8 * N^2 per replica (k+1 rows read, one written);
+    gossip round: 2 * 8 * N^2 per replica (every view entry read once and written once; the
+    k+1 readers of a row share it through L2 because the merge walks the matrix by column panels);
     request path: 8 B record + 26 B result, plus a 256 B view window per request that offloads."""
     st = wl.settings
-    gossip_round = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
+    gossip_round = 2 * 8 * st.n_peers ** 2 * st.n_replicas
     offloaded = stats_delta["n_delegated"] + stats_delta["n_fallback_local"] + stats_delta["n_failed"]
     req = stats_delta["n_requests"] * (8 + 26) + offloaded * 256
     return gossip_round, req
@@ -186,6 +187,8 @@ def run_gpu(args):
                 "ms_per_launch": t * 1e3}
 
     roof_merge = roof("k_gossip_merge", g_bytes)
+    if roof_merge:      # context: bytes a merge without L2 reuse would move (k+1 rows read, one written)
+        roof_merge["bytes_per_launch_without_reuse"] = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
     roof_req = roof("k_step_fused", req_bytes / max(1, prof.get("k_step_fused", (0, 1))[1]))
     roofline = roof_merge if dom == "k_gossip_merge" else roof_req
 

@@ -1,5 +1,7 @@
 // Gossip round: churn + self entries + partner choice (per peer), row merge (streaming
 // 64-bit max over gathered rows), and the scattered single-entry updates.
+#include <cstdlib>
+
 #include "wwws_internal.cuh"
 
 namespace wwws {
@@ -42,65 +44,94 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
     *reinterpret_cast<int4*>(n.partner + x * 4) = make_int4(part[0], part[1], part[2], part[3]);
 }
 
-// Streaming merge.  One block handles `kTile` consecutive columns of one row: new row =
-// max(old row, rows of the partners that answered).  16-byte vector accesses; the partner
-// rows are independent loads, so each thread keeps (1+k) * kUnroll loads in flight.
+// Streaming merge: new row = max(old row, rows of the partners that answered).
+//
+// A row is read by its owner and by every node that pulls it (k+1 readers on average), so the
+// order of the work decides how often it comes from HBM.  The matrix is cut into column panels
+// narrow enough that one panel of all N rows stays in L2 (N * panel_cols * 8 bytes); blocks are
+// numbered panel-major, so the blocks in flight at any time work on the same panel: the first
+// reader of a row segment brings it in from HBM, the others hit L2.  HBM traffic per round drops
+// from (k+2) * 8 * N^2 towards 2 * 8 * N^2 (each entry read once, written once).  Stores are
+// streaming (evict-first) so that they do not push the panel out.
+//
+// A thread moves 32 bytes (four entries) per row it touches: one 256-bit load per source row.
 constexpr int kMergeThreads = 256;
-constexpr int kUnroll = 2;
-constexpr int kTile = kMergeThreads * 2 * kUnroll;   // columns per block
+constexpr int kMergeIters = 4;                         // rows per thread
+constexpr int kMergeMaxRows = 128;                     // rows per block at the narrowest panel
 
-__device__ __forceinline__ ulonglong2 ld16(const uint64_t* p)
+struct Q4 { uint64_t a, b, c, d; };                    // four entries = 32 bytes
+
+__device__ __forceinline__ Q4 ld32(const char* p)
 {
-    ulonglong2 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v2.u64 {%0,%1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p));
+    Q4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u64 {%0,%1,%2,%3}, [%4];"
+                 : "=l"(v.a), "=l"(v.b), "=l"(v.c), "=l"(v.d) : "l"(p));
     return v;
 }
-__device__ __forceinline__ void st16(uint64_t* p, ulonglong2 v)
+__device__ __forceinline__ void st32_stream(char* p, const Q4& v)
 {
-    asm volatile("st.global.L1::no_allocate.v2.u64 [%0], {%1,%2};" ::"l"(p), "l"(v.x), "l"(v.y) : "memory");
+    asm volatile("st.global.cs.v4.u64 [%0], {%1,%2,%3,%4};" ::"l"(p), "l"(v.a), "l"(v.b), "l"(v.c), "l"(v.d) : "memory");
 }
 __device__ __forceinline__ uint64_t umax64(uint64_t a, uint64_t b) { return a > b ? a : b; }
-
-__global__ void __launch_bounds__(kMergeThreads) k_gossip_merge(Net n, uint32_t tiles_per_row)
+__device__ __forceinline__ void join(Q4& x, const Q4& y)
 {
-    const uint64_t blk = uint64_t(blockIdx.y) * gridDim.x + blockIdx.x;   // over Rp * N * tiles_per_row
-    const uint64_t rowid = blk / tiles_per_row;                             // r * N + i
-    if (rowid >= uint64_t(n.Rp) * n.N) return;
-    const uint32_t tile = uint32_t(blk - rowid * tiles_per_row);
-    const uint32_t r = uint32_t(rowid / n.N);
-    const uint64_t* src[4];
-    int ns = 0;
-    if (n.online[rowid]) {
-        const int4 p4 = *reinterpret_cast<const int4*>(n.partner + rowid * 4);
-        const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
-#pragma unroll
-        for (int s = 0; s < 4; ++s)
-            if (p[s] >= 0 && n.online[size_t(r) * n.N + p[s]]) src[ns++] = n.view + (size_t(r) * n.N + p[s]) * n.ld;
-    }
-    const uint64_t* own = n.view + rowid * n.ld;
-    uint64_t* out = n.view_new + rowid * n.ld;
-    const uint32_t c0 = tile * kTile + threadIdx.x * 2;
-    ulonglong2 acc[kUnroll];
-    bool live[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const uint32_t c = c0 + u * kMergeThreads * 2;
-        live[u] = c < n.ld;
-        acc[u] = live[u] ? ld16(own + c) : make_ulonglong2(0, 0);
-    }
-    for (int s = 0; s < ns; ++s) {
-        ulonglong2 v[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const uint32_t c = c0 + u * kMergeThreads * 2;
-            v[u] = live[u] ? ld16(src[s] + c) : make_ulonglong2(0, 0);
+    x.a = umax64(x.a, y.a); x.b = umax64(x.b, y.b); x.c = umax64(x.c, y.c); x.d = umax64(x.d, y.d);
+}
+
+// grid.x runs over (replica, panel, row group).  A thread owns one 32-byte column chunk of the
+// panel and walks kMergeIters rows of the block's row group.  Prologue: every row of the group
+// resolves its sources once (partner rows that answered, -1 otherwise) into shared memory, so
+// the streaming part has no dependent metadata loads.
+__global__ void __launch_bounds__(kMergeThreads, 4) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
+                                                                     uint32_t n_panels, uint32_t groups_per_panel)
+{
+    __shared__ int4 s_src[kMergeMaxRows];
+    const uint32_t b = blockIdx.x;
+    const uint32_t per_replica = n_panels * groups_per_panel;
+    const uint32_t r = b / per_replica;
+    const uint32_t rem = b - r * per_replica;
+    const uint32_t panel = rem / groups_per_panel, group = rem - panel * groups_per_panel;
+    const uint32_t rstep = kMergeThreads >> chunk_shift;                  // rows covered by one pass of the block
+    const uint32_t rows_per_block = rstep * kMergeIters;
+    const uint32_t row0 = group * rows_per_block;
+    const size_t rbase = size_t(r) * n.N;
+    if (threadIdx.x < rows_per_block) {
+        int4 src = make_int4(-1, -1, -1, -1);
+        const uint32_t row = row0 + threadIdx.x;
+        if (row < n.N && n.online[rbase + row]) {
+            const int4 p4 = *reinterpret_cast<const int4*>(n.partner + (rbase + row) * 4);
+            const uint8_t* on = n.online + rbase;
+            src.x = p4.x >= 0 && on[p4.x] ? p4.x : -1;
+            src.y = p4.y >= 0 && on[p4.y] ? p4.y : -1;
+            src.z = p4.z >= 0 && on[p4.z] ? p4.z : -1;
+            src.w = p4.w >= 0 && on[p4.w] ? p4.w : -1;
         }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) { acc[u].x = umax64(acc[u].x, v[u].x); acc[u].y = umax64(acc[u].y, v[u].y); }
+        s_src[threadIdx.x] = src;
     }
+    __syncthreads();
+    const uint32_t c = panel * panel_cols + 4u * (threadIdx.x & ((1u << chunk_shift) - 1u));
+    if (c >= n.ld) return;
+    const uint32_t ld8 = n.ld * 8u;
+    const char* in = reinterpret_cast<const char*>(n.view + rbase * n.ld + c);
+    char* out = reinterpret_cast<char*>(n.view_new + rbase * n.ld + c);
+    uint32_t lr = threadIdx.x >> chunk_shift;
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u)
-        if (live[u]) st16(out + c0 + u * kMergeThreads * 2, acc[u]);
+    for (int it = 0; it < kMergeIters; ++it, lr += rstep) {
+        const uint32_t row = row0 + lr;
+        if (row >= n.N) break;
+        const int4 src = s_src[lr];
+        Q4 acc = ld32(in + uint64_t(row) * ld8);
+        Q4 v0, v1, v2, v3;
+        if (src.x >= 0) v0 = ld32(in + uint64_t(uint32_t(src.x)) * ld8);
+        if (src.y >= 0) v1 = ld32(in + uint64_t(uint32_t(src.y)) * ld8);
+        if (src.z >= 0) v2 = ld32(in + uint64_t(uint32_t(src.z)) * ld8);
+        if (src.w >= 0) v3 = ld32(in + uint64_t(uint32_t(src.w)) * ld8);
+        if (src.x >= 0) join(acc, v0);
+        if (src.y >= 0) join(acc, v1);
+        if (src.z >= 0) join(acc, v2);
+        if (src.w >= 0) join(acc, v3);
+        st32_stream(out + uint64_t(row) * ld8, acc);
+    }
 }
 
 // The three single-entry updates of a round, all joins (max), applied after the row merge:
@@ -129,15 +160,33 @@ __global__ void k_gossip_fixup(Net n)
     if (marks) atomicAdd(&n.stats[size_t(r) * sCount + sOfflineMarks], (unsigned long long)marks);
 }
 
+// Panel width: the widest power of two (32 .. 1024 columns) whose panel of N rows fits the
+// L2 budget; WWWS_PANEL_BYTES overrides the budget (tuning).
+static uint32_t panel_columns(const Net& n)
+{
+    static const uint64_t budget = [] {
+        const char* e = getenv("WWWS_PANEL_BYTES");
+        const uint64_t v = e ? strtoull(e, nullptr, 10) : 0;
+        return v ? v : (16ull << 20);
+    }();
+    uint32_t pc = 1024;
+    while (pc > 32 && uint64_t(n.N) * pc * 8 > budget) pc >>= 1;
+    return pc;
+}
+
 void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c)
 {
     const dim3 pg((n.N + 127) / 128, n.Rp);
     { Timed t(c, kGossipPeer); k_gossip_peer<<<pg, 128, 0, c.stream>>>(n, round); }
-    const uint32_t tiles = (n.ld + kTile - 1) / kTile;
-    const uint64_t blocks = uint64_t(n.Rp) * n.N * tiles;
-    const uint32_t gx = blocks > 65535u * 32u ? 65535u * 32u : uint32_t(blocks);   // x up to 2^31-1; keep y small
-    const uint32_t gy = uint32_t((blocks + gx - 1) / gx);
-    { Timed t(c, kGossipMerge); k_gossip_merge<<<dim3(gx, gy), kMergeThreads, 0, c.stream>>>(n, tiles); }
+    const uint32_t pc = panel_columns(n);
+    uint32_t shift = 0;
+    while ((4u << shift) < pc) ++shift;                                   // 32-byte chunks per row segment = pc / 4
+    const uint32_t rows_per_block = (kMergeThreads >> shift) * kMergeIters;
+    const uint32_t n_panels = (n.ld + pc - 1) / pc;
+    const uint32_t groups = (n.N + rows_per_block - 1) / rows_per_block;
+    const uint64_t blocks = uint64_t(n.Rp) * n_panels * groups;
+    { Timed t(c, kGossipMerge);
+      k_gossip_merge<<<uint32_t(blocks), kMergeThreads, 0, c.stream>>>(n, pc, shift, n_panels, groups); }
     { Timed t(c, kGossipFixup); k_gossip_fixup<<<pg, 128, 0, c.stream>>>(n); }
 }
 
