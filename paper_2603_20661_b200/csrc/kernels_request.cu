@@ -1,35 +1,10 @@
 // Per-request kernels: dispatch, duel-and-judge, settlement, and the fused step.
 // One warp owns one request; lane c owns candidate c of the request's 32-peer window.
-#include "wwws_internal.cuh"
+#include "request_common.cuh"
 
 namespace wwws {
 
 constexpr int kWarpsPerBlock = 8;
-constexpr unsigned kFull = 0xffffffffu;
-
-// ---- per-block counters -------------------------------------------------------------------
-
-struct BlockStats {
-    unsigned long long c[sCount];
-};
-
-__device__ __forceinline__ void stats_begin(BlockStats& s)
-{
-    if (threadIdx.x < sCount) s.c[threadIdx.x] = 0;
-    __syncthreads();
-}
-__device__ __forceinline__ void stats_add(BlockStats& s, uint32_t k, unsigned long long v)
-{
-    if (v) atomicAdd(&s.c[k], v);
-}
-__device__ __forceinline__ void stats_end(const Net& n, BlockStats& s, uint32_t r)
-{
-    __syncthreads();
-    if (threadIdx.x < sCount) {
-        const unsigned long long v = s.c[threadIdx.x];
-        if (v) atomicAdd(&n.stats[size_t(r) * sCount + threadIdx.x], v);
-    }
-}
 
 // ---- the candidate window of one request, spread over a warp -------------------------------
 
@@ -42,47 +17,13 @@ struct Window {
     Rnd4 y; uint32_t y_slot;       // cached draw pair
 };
 
-// D3: the block of the id ring this request samples from.
-__device__ __forceinline__ uint32_t pick_block(const Net& n, uint32_t o, uint32_t w2)
-{
-    uint32_t rank;
-    if (n.rank_cdf) {
-        uint32_t lo = 0, hi = n.n_rank;           // first index with w2 < cdf[idx]
-        while (lo < hi) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (w2 < __ldg(n.rank_cdf + mid)) hi = mid; else lo = mid + 1;
-        }
-        rank = lo > n.n_blk - 1 ? n.n_blk - 1 : lo;
-    } else {
-        rank = below(w2, n.n_blk);
-    }
-    return (o / kWin + rank) % n.n_blk;
-}
-
-// D4: fp32 score and integer weight of this lane's candidate.  Every fp32 operation is an
-// explicitly rounded IEEE operation (no fused multiply-add), so a CPU computing the same
-// expression in binary32 gets the same bits.
+// D4 for this lane's candidate.
 __device__ __forceinline__ void score_lane(const Net& n, Window& w, uint32_t lane)
 {
-    w.W = 0; w.score = 0.0f;
     const uint32_t id = kWin * w.blk + lane;
-    const size_t rowx = size_t(w.r) * n.N + w.o;
-    const uint64_t e = n.view[rowx * n.ld + id];              // id < ld always: coalesced 256 B per warp
-    if (id >= n.N || id == w.o || e == 0 || (e & kOffBit)) return;
-    const uint32_t advcap = uint32_t(e >> 20) & kCapMax, advq = uint32_t(e) & kQMax;
-    const float wl = n.w_led[size_t(w.r) * n.N + id];
-    if (!(wl > 0.0f) || advcap == 0) return;
-    float spare = 1.0f;
-    if (n.flags & 2u) {
-        const float utilf = __fdiv_rn(__uint2float_rn(advq * 16u), __fmul_rn(__uint2float_rn(advcap), n.uwf));
-        spare = __fsub_rn(1.0f, utilf);
-        if (!(spare > 0.0f)) spare = 0.0f;
-    }
-    const float score = __fmul_rn(wl, spare);
-    const float scaled = __fmul_rn(score, 256.0f);
-    const uint64_t W = scaled >= 72057594037927936.0f ? (1ull << 56) : __float2ull_rz(scaled);
-    w.W = W;
-    w.score = W ? score : 0.0f;
+    const uint64_t e = n.view[(size_t(w.r) * n.N + w.o) * n.ld + id];     // id < ld always: coalesced 256 B per warp
+    const float wl = id < n.N ? n.w_led[size_t(w.r) * n.N + id] : 0.0f;
+    w.W = candidate_weight(n, w.o, id, e, wl, w.score);
 }
 
 __device__ __forceinline__ uint64_t warp_incl_scan(uint64_t v, uint32_t lane)
@@ -136,19 +77,6 @@ __device__ __forceinline__ int find_executor(const Net& n, Window& w, uint32_t l
     return -1;
 }
 
-// Origin side of dispatch (D1, D2).  Returns 1 if the request goes to the network, else
-// writes the local / dropped / failed code to `code`.
-__device__ __forceinline__ bool origin_offloads(const Net& n, uint32_t r, uint32_t o, const Rnd4& rx, int& code)
-{
-    if (o >= n.N) { set_error(n, eArg, o); code = -3; return false; }
-    const size_t ox = size_t(r) * n.N + o;
-    if (!n.online[ox]) { code = -3; return false; }
-    const uint32_t cap = n.cap_eff[ox];
-    code = cap == 0 ? -4 : -1;
-    return util_at_least(cap, n.backlog[ox], n.util_window_ms, n.offload_util_pm[ox]) &&
-           ppm(rx.w[0]) < n.offload_ppm[ox] && n.credit[ox] >= n.R;
-}
-
 // J2 + J3 for a delegated request flagged as a duel.  Returns the outcome code.
 __device__ __forceinline__ uint32_t run_duel(const Net& n, Window& w, uint32_t lane, int a, int& b, int (&jd)[4])
 {
@@ -172,87 +100,6 @@ __device__ __forceinline__ uint32_t run_duel(const Net& n, Window& w, uint32_t l
         votes_a += va;
     }
     return 2 * votes_a > nj ? 1u : (2 * votes_a < nj ? 2u : 3u);
-}
-
-// ---- settlement of one request (one thread) ----------------------------------------------------
-
-__device__ __forceinline__ void add64(long long* p, long long v) { atomicAdd((unsigned long long*)p, (unsigned long long)v); }
-
-struct SettleAcc {
-    uint32_t c[sSumLat];           // counters before sSumLat are small
-    unsigned long long sum_lat;
-};
-
-__device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t o, uint32_t li, uint32_t lo, int a, int b,
-                                           const int (&jd)[4], uint32_t oc, bool near, SettleAcc& s)
-{
-    const size_t base = size_t(r) * n.N;
-    const uint64_t work = uint64_t(li) + lo;
-    s.c[sRequests]++;
-    if (near) s.c[sNear]++;
-    if (a == -3) { s.c[sDropped]++; return; }
-    if (a == -4) { s.c[sFailed]++; return; }
-    uint32_t ex;
-    if (a < 0) {
-        s.c[a == -1 ? sLocal : sFallback]++;
-        add64(&n.d_backlog[base + o], (long long)work);
-        atomicAdd(&n.served_local[base + o], 1ull);
-        ex = o;
-    } else {
-        s.c[sDelegated]++;
-        long long pay = n.R;
-        add64(&n.d_credit[base + a], n.R);
-        add64(&n.d_backlog[base + a], (long long)work);
-        atomicAdd(&n.served[base + a], 1ull);
-        ex = uint32_t(a);
-        if (oc != 0) s.c[sDuel]++;
-        if (oc == 4) s.c[sDuelCancelled]++;
-        if (oc >= 1 && oc <= 3) {
-            pay += n.R;
-            add64(&n.d_credit[base + b], n.R);
-            add64(&n.d_backlog[base + b], (long long)work);
-            atomicAdd(&n.served[base + b], 1ull);
-            atomicAdd(&n.d_duels[base + a], 1u);
-            atomicAdd(&n.d_duels[base + b], 1u);
-            int nj = 0;
-#pragma unroll
-            for (int l = 0; l < 4; ++l)
-                if (jd[l] >= 0) { add64(&n.d_backlog[base + jd[l]], (long long)(uint64_t(li) + 2ull * lo)); ++nj; }
-            s.c[sJudgeEvals] += nj;
-            if (oc == 3) s.c[sDraw]++;
-            else {
-                const int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
-                const long long pot = n.P - n.R_add, share = pot / nj;
-                add64(&n.d_credit[base + lose], -n.P);
-                add64(&n.d_credit[base + win], n.R_add + (pot - share * nj));
-                atomicAdd(&n.d_wins[base + win], 1u);
-#pragma unroll
-                for (int l = 0; l < 4; ++l)
-                    if (jd[l] >= 0) add64(&n.d_credit[base + jd[l]], share);
-            }
-        }
-        add64(&n.d_credit[base + o], -pay);
-    }
-    const uint64_t cap = n.cap_eff[base + ex];
-    const uint64_t t = (uint64_t(n.backlog[base + ex]) + work) * 1000ull, tq = t / cap;
-    const uint64_t lat = tq + (tq * cap != t ? 1 : 0) + (a >= 0 ? n.hop_ms : 0);
-    const uint64_t ideal = (work * 1000ull + n.cap_ref - 1) / n.cap_ref;
-    const uint64_t deadline = uint64_t(n.slo_num) * ideal / n.slo_den;
-    s.sum_lat += lat;
-    if (lat <= deadline) s.c[sSloMet]++;
-}
-
-__device__ __forceinline__ void acc_zero(SettleAcc& s)
-{
-#pragma unroll
-    for (int k = 0; k < int(sSumLat); ++k) s.c[k] = 0;
-    s.sum_lat = 0;
-}
-__device__ __forceinline__ void acc_flush(BlockStats& bs, const SettleAcc& s)
-{
-#pragma unroll
-    for (int k = 0; k < int(sSumLat); ++k) stats_add(bs, k, s.c[k]);
-    stats_add(bs, sSumLat, s.sum_lat);
 }
 
 // ---- kernels ---------------------------------------------------------------------------------
@@ -363,52 +210,6 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
     stats_end(n, bs, r);
 }
 
-// Dispatch + duel-and-judge + settlement of one request in one pass.  Legal because every
-// update goes to a pending column (d_credit, d_wins, d_duels, d_backlog) or a counter, while
-// all decisions read the state as it stood when the batch started.
-__global__ void __launch_bounds__(kWarpsPerBlock * 32) k_step_fused(Net n, uint64_t first, uint32_t count)
-{
-    __shared__ BlockStats bs;
-    stats_begin(bs);
-    const uint32_t lane = threadIdx.x & 31, r = blockIdx.y;
-    const uint32_t idx = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
-    if (idx < count) {
-        const uint64_t q = first + idx;
-        const size_t x = size_t(r) * n.Q + q;
-        Window w;
-        w.r = r; w.rg = r + n.replica_offset; w.q = uint32_t(q); w.o = n.origin[x];
-        w.n_draws = 0; w.n_probes = 0; w.near = false; w.y_slot = 0xffffffffu; w.W = 0; w.score = 0.0f; w.blk = 0;
-        const Rnd4 rx = draw(n, w.q, 0, w.rg, kOrigin);
-        int a, b = -1, jd[4] = { -1, -1, -1, -1 };
-        uint32_t oc = 0;
-        float sa = 0.0f, ssum = 0.0f;
-        if (origin_offloads(n, r, w.o, rx, a)) {
-            const int local_code = a;
-            w.blk = pick_block(n, w.o, rx.w[2]);
-            score_lane(n, w, lane);
-            if (n.score_sum) {
-                for (int l = 0; l < 32; ++l) ssum = __fadd_rn(ssum, __shfl_sync(kFull, w.score, l));
-            }
-            a = find_executor(n, w, lane);
-            if (a >= 0) {
-                sa = __shfl_sync(kFull, w.score, a & 31);
-                if (ppm(rx.w[1]) < n.p_duel) oc = run_duel(n, w, lane, a, b, jd);
-            } else a = local_code == -4 ? -4 : -2;
-        }
-        if (lane == 0) {
-            n.exec_a[x] = a; n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = w.near ? 1 : 0;
-            *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
-            if (n.score_a) n.score_a[x] = sa;
-            if (n.score_sum) n.score_sum[x] = ssum;
-            SettleAcc s; acc_zero(s);
-            s.c[sProbes] = w.n_probes;
-            settle_one(n, r, w.o, n.len_in[x], n.len_out[x], a, b, jd, oc, w.near, s);
-            acc_flush(bs, s);
-        }
-    }
-    stats_end(n, bs, r);
-}
-
 static dim3 warp_grid(const Net& n, uint32_t count) { return dim3((count + kWarpsPerBlock - 1) / kWarpsPerBlock, n.Rp); }
 
 void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
@@ -426,10 +227,4 @@ void launch_settle(const Net& n, uint64_t first, uint32_t count, const LaunchCtx
     Timed t(c, kSettle);
     k_settle<<<dim3((count + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, first, count);
 }
-void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
-{
-    Timed t(c, kStepFused);
-    k_step_fused<<<warp_grid(n, count), kWarpsPerBlock * 32, 0, c.stream>>>(n, first, count);
-}
-
 }  // namespace wwws

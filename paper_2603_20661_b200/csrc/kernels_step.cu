@@ -1,0 +1,241 @@
+// The fused step kernel: dispatch + duel-and-judge + settlement, one thread per request.
+//
+// Fusing is legal because every update of a batch goes to a pending column (d_credit, d_wins,
+// d_duels, d_backlog) or a counter, while all decisions read the state as it stood when the
+// batch started.
+//
+// A thread scores its request's 32 candidates serially (the window is 256 contiguous bytes of
+// the origin's view row: eight 32-byte loads) and keeps the integer weights in shared memory,
+// laid out [candidate][slot] so that lanes never conflict and so that ANY thread of the block
+// can continue a request.  That is used for the duels: only a few requests per block become
+// duels, so instead of letting every warp run the long duel code for one or two of its lanes,
+// duel requests are queued in shared memory and picked up densely by the first threads of the
+// block after a barrier.
+#include "request_common.cuh"
+
+namespace wwws {
+
+template <int BT> struct StepShared {
+    unsigned long long W[kWin][BT];      // integer weights, 0 = not in play
+    BlockStats stats;
+    uint32_t n_duel;
+    uint16_t queue[BT];                  // slots whose request became a duel
+    struct Ctx { int32_t a; uint32_t blk; uint32_t draws_probes_near; } ctx[BT];
+};
+
+// Draw state of one request, held by the thread that is working on it.
+struct Draws {
+    uint64_t G0, G1, G2, G3;             // sums of the four 8-candidate groups still in play
+    uint32_t n_draws, n_probes;
+    bool near;
+    Rnd4 y; uint32_t y_slot;
+};
+
+// D5: one draw proportional to the weights still in play, by integer prefix sums: first the
+// 8-candidate group, then the candidate inside it.  Returns the candidate or -1 if none is left.
+template <int BT>
+__device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, uint32_t slot, Draws& d, uint32_t q, uint32_t rg)
+{
+    const uint64_t S = d.G0 + d.G1 + d.G2 + d.G3;
+    if (S == 0) return -1;
+    const uint32_t k = d.n_draws++;
+    if (d.y_slot != (k >> 1)) { d.y = draw(n, q, k >> 1, rg, kDraw); d.y_slot = k >> 1; }
+    const uint64_t u = (k & 1u) ? (uint64_t(d.y.w[2]) << 32 | d.y.w[3]) : (uint64_t(d.y.w[0]) << 32 | d.y.w[1]);
+    const uint64_t r64 = __umul64hi(u, S);
+    uint64_t lo = 0;
+    int g = 0;
+    if (r64 >= lo + d.G0) { lo += d.G0; g = 1;
+        if (r64 >= lo + d.G1) { lo += d.G1; g = 2;
+            if (r64 >= lo + d.G2) { lo += d.G2; g = 3; } } }
+    int pick = -1;
+    uint64_t wp = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint64_t w = sh.W[8 * g + j][slot];
+        if (pick < 0) {
+            if (r64 < lo + w) { pick = 8 * g + j; wp = w; }
+            else lo += w;
+        }
+    }
+    const uint64_t m1 = r64 - lo, m2 = lo + wp - 1 - r64;
+    if ((m1 < m2 ? m1 : m2) <= S / 100000ull) d.near = true;
+    sh.W[pick][slot] = 0;
+    if (g == 0) d.G0 -= wp; else if (g == 1) d.G1 -= wp; else if (g == 2) d.G2 -= wp; else d.G3 -= wp;
+    return pick;
+}
+
+// D6: the drawn candidate answers by its true state and its own accept policy.
+__device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg, uint32_t q, uint32_t blk, int pick)
+{
+    const size_t x = size_t(r) * n.N + kWin * blk + pick;
+    const uint32_t cap = n.cap_eff[x];
+    if (!n.online[x] || cap == 0) return false;
+    if (util_at_least(cap, n.backlog[x], n.util_window_ms, n.accept_util_pm[x])) return false;
+    return ppm(draw(n, q, uint32_t(pick) >> 2, rg, kProbe).w[pick & 3]) < n.accept_ppm[x];
+}
+
+template <int BT>
+__device__ __forceinline__ int find_peer(const Net& n, StepShared<BT>& sh, uint32_t slot, Draws& d, uint32_t r, uint32_t rg,
+                                         uint32_t q, uint32_t blk)
+{
+    while (d.n_probes < n.max_probes) {
+        const int pick = draw_candidate(n, sh, slot, d, q, rg);
+        if (pick < 0) break;
+        d.n_probes++;
+        if (probe_peer(n, r, rg, q, blk, pick)) return int(kWin * blk + pick);
+    }
+    return -1;
+}
+
+template <int BT>
+__global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32_t count)
+{
+    __shared__ StepShared<BT> sh;
+    stats_begin(sh.stats);                       // barrier inside
+    if (threadIdx.x == 0) sh.n_duel = 0;
+    __syncthreads();
+    const uint32_t r = blockIdx.y, rg = r + n.replica_offset;
+    const uint32_t slot = threadIdx.x;
+    const uint32_t idx = blockIdx.x * BT + slot;
+    SettleAcc acc; acc_zero(acc);
+
+    // ---- dispatch (D1..D6), one request per thread -----------------------------------------
+    if (idx < count) {
+        const uint32_t q = uint32_t(first + idx);
+        const size_t x = size_t(r) * n.Q + first + idx;
+        const uint32_t o = n.origin[x];
+        const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
+        int a;
+        float sa = 0.0f, ssum = 0.0f;
+        Draws d;
+        d.G0 = d.G1 = d.G2 = d.G3 = 0; d.n_draws = 0; d.n_probes = 0; d.near = false; d.y_slot = 0xffffffffu;
+        uint32_t blk = 0;
+        bool duel = false;
+        if (origin_offloads(n, r, o, rx, a)) {
+            const int local_code = a;
+            blk = pick_block(n, o, rx.w[2]);
+            const uint64_t* win = n.view + (size_t(r) * n.N + o) * n.ld + kWin * blk;
+            const float* wled = n.w_led + size_t(r) * n.N;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint64_t gsum = 0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int c0 = 8 * g + 4 * h;
+                    const ulonglong4 e4 = *reinterpret_cast<const ulonglong4*>(win + c0);     // 32 B of the window
+                    const uint64_t e[4] = { e4.x, e4.y, e4.z, e4.w };
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t id = kWin * blk + c0 + j;
+                        const float wl = id < n.N ? wled[id] : 0.0f;
+                        float sc;
+                        const uint64_t W = candidate_weight(n, o, id, e[j], wl, sc);
+                        sh.W[c0 + j][slot] = W;
+                        gsum += W;
+                        ssum = __fadd_rn(ssum, sc);                                            // lane-ascending fp32 sum
+                    }
+                }
+                if (g == 0) d.G0 = gsum; else if (g == 1) d.G1 = gsum; else if (g == 2) d.G2 = gsum; else d.G3 = gsum;
+            }
+            a = find_peer<BT>(n, sh, slot, d, r, rg, q, blk);
+            if (a >= 0) {
+                if (n.score_a) {
+                    float sc;
+                    candidate_weight(n, o, uint32_t(a), win[a & 31], wled[a], sc);
+                    sa = sc;
+                }
+                duel = ppm(rx.w[1]) < n.p_duel;
+            } else a = local_code == -4 ? -4 : -2;
+        }
+        n.exec_a[x] = a;
+        if (n.score_a) n.score_a[x] = sa;
+        if (n.score_sum) n.score_sum[x] = ssum;
+        if (duel) {
+            const uint32_t k = atomicAdd(&sh.n_duel, 1u);
+            sh.queue[k] = uint16_t(slot);
+            sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
+            sh.ctx[slot].draws_probes_near = d.n_draws | (d.n_probes << 8) | (d.near ? 1u << 16 : 0u);
+        } else {
+            n.exec_b[x] = -1; n.outcome[x] = 0; n.rflags[x] = d.near ? 1 : 0;
+            *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(-1, -1, -1, -1);
+            const int jd[4] = { -1, -1, -1, -1 };
+            acc.c[sProbes] += d.n_probes;
+            settle_one(n, r, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
+        }
+    }
+    __syncthreads();
+
+    // ---- duel-and-judge (J2, J3) for the queued requests, densely -----------------------------
+    if (threadIdx.x < sh.n_duel) {
+        const uint32_t ds = sh.queue[threadIdx.x];
+        const uint32_t didx = blockIdx.x * BT + ds;
+        const uint32_t q = uint32_t(first + didx);
+        const size_t x = size_t(r) * n.Q + first + didx;
+        const int a = sh.ctx[ds].a;
+        const uint32_t blk = sh.ctx[ds].blk, packed = sh.ctx[ds].draws_probes_near;
+        Draws d;
+        d.n_draws = packed & 0xffu; d.n_probes = (packed >> 8) & 0xffu; d.near = (packed >> 16) & 1u; d.y_slot = 0xffffffffu;
+        uint64_t gs[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            gs[g] = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) gs[g] += sh.W[8 * g + j][ds];
+        }
+        d.G0 = gs[0]; d.G1 = gs[1]; d.G2 = gs[2]; d.G3 = gs[3];
+        int b = find_peer<BT>(n, sh, ds, d, r, rg, q, blk);
+        int jd[4] = { -1, -1, -1, -1 };
+        uint32_t oc = 4;
+        if (b >= 0) {
+            int nj = 0;
+            while (nj < int(n.n_judges)) {
+                const int pick = draw_candidate(n, sh, ds, d, q, rg);
+                if (pick < 0) break;
+                const int id = int(kWin * blk + pick);
+                if (n.online[size_t(r) * n.N + id]) {
+                    if (nj == 0) jd[0] = id; else if (nj == 1) jd[1] = id; else if (nj == 2) jd[2] = id; else jd[3] = id;
+                    ++nj;
+                }
+            }
+            if (nj == 0) b = -1;
+            else {
+                const uint64_t thr = ((1ull << 32) + n.quality[size_t(r) * n.N + a] - n.quality[size_t(r) * n.N + b]) >> 1;
+                int votes_a = 0;
+                for (int l = 0; l < nj; ++l) {
+                    const Rnd4 y = draw(n, q, uint32_t(l), rg, kJudge);
+                    bool va = uint64_t(y.w[0]) < thr;
+                    if (ppm(y.w[1]) < n.p_noise) va = !va;
+                    votes_a += va;
+                }
+                oc = 2 * votes_a > nj ? 1u : (2 * votes_a < nj ? 2u : 3u);
+            }
+        }
+        n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = d.near ? 1 : 0;
+        *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
+        acc.c[sProbes] += d.n_probes;
+        settle_one(n, r, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
+    }
+
+    // ---- counters: warp reduce, block reduce, one atomic per counter and block ---------------
+#pragma unroll
+    for (int k = 0; k < int(sSumLat); ++k) {
+        const uint32_t v = __reduce_add_sync(kFull, acc.c[k]);
+        if ((threadIdx.x & 31) == 0) stats_add(sh.stats, k, v);
+    }
+    unsigned long long sl = acc.sum_lat;
+    for (int o = 16; o; o >>= 1) sl += __shfl_down_sync(kFull, sl, o);
+    if ((threadIdx.x & 31) == 0) stats_add(sh.stats, sSumLat, sl);
+    stats_end(n, sh.stats, r);
+}
+
+void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    Timed t(c, kStepFused);
+    // small batches: small blocks, so that the requests spread over all SMs
+    if (uint64_t(count) * n.Rp >= 148ull * 128 * 4)
+        k_step_fused<128><<<dim3((count + 127) / 128, n.Rp), 128, 0, c.stream>>>(n, first, count);
+    else
+        k_step_fused<32><<<dim3((count + 31) / 32, n.Rp), 32, 0, c.stream>>>(n, first, count);
+}
+
+}  // namespace wwws

@@ -1,0 +1,168 @@
+// Pieces of the request path shared by the warp-per-request kernels (dispatch, duel, settle)
+// and the thread-per-request fused step.
+#pragma once
+#include "wwws_internal.cuh"
+
+namespace wwws {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+// ---- per-block counters -------------------------------------------------------------------
+
+struct BlockStats {
+    unsigned long long c[sCount];
+};
+
+__device__ __forceinline__ void stats_begin(BlockStats& s)
+{
+    if (threadIdx.x < sCount) s.c[threadIdx.x] = 0;
+    __syncthreads();
+}
+__device__ __forceinline__ void stats_add(BlockStats& s, uint32_t k, unsigned long long v)
+{
+    if (v) atomicAdd(&s.c[k], v);
+}
+__device__ __forceinline__ void stats_end(const Net& n, BlockStats& s, uint32_t r)
+{
+    __syncthreads();
+    if (threadIdx.x < sCount) {
+        const unsigned long long v = s.c[threadIdx.x];
+        if (v) atomicAdd(&n.stats[size_t(r) * sCount + threadIdx.x], v);
+    }
+}
+
+// D3: the block of the id ring this request samples from.
+__device__ __forceinline__ uint32_t pick_block(const Net& n, uint32_t o, uint32_t w2)
+{
+    uint32_t rank;
+    if (n.rank_cdf) {
+        uint32_t lo = 0, hi = n.n_rank;           // first index with w2 < cdf[idx]
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (w2 < __ldg(n.rank_cdf + mid)) hi = mid; else lo = mid + 1;
+        }
+        rank = lo > n.n_blk - 1 ? n.n_blk - 1 : lo;
+    } else {
+        rank = below(w2, n.n_blk);
+    }
+    return (o / kWin + rank) % n.n_blk;
+}
+
+// D4: fp32 score and integer weight of candidate `id` as the origin `o` sees it: view entry `e`
+// of the origin's row, ledger weight `wl`.  Every fp32 operation is an explicitly rounded IEEE
+// operation (no fused multiply-add), so a CPU computing the same expression in binary32 gets the
+// same bits.  Returns the weight (0 = not eligible) and the score through `score`.
+__device__ __forceinline__ uint64_t candidate_weight(const Net& n, uint32_t o, uint32_t id, uint64_t e, float wl, float& score)
+{
+    score = 0.0f;
+    if (id >= n.N || id == o || e == 0 || (e & kOffBit)) return 0;
+    const uint32_t advcap = uint32_t(e >> 20) & kCapMax, advq = uint32_t(e) & kQMax;
+    if (!(wl > 0.0f) || advcap == 0) return 0;
+    float spare = 1.0f;
+    if (n.flags & 2u) {
+        const float utilf = __fdiv_rn(__uint2float_rn(advq * 16u), __fmul_rn(__uint2float_rn(advcap), n.uwf));
+        spare = __fsub_rn(1.0f, utilf);
+        if (!(spare > 0.0f)) spare = 0.0f;
+    }
+    const float sc = __fmul_rn(wl, spare);
+    const float scaled = __fmul_rn(sc, 256.0f);
+    const uint64_t W = scaled >= 72057594037927936.0f ? (1ull << 56) : __float2ull_rz(scaled);
+    if (W) score = sc;
+    return W;
+}
+
+// Origin side of dispatch (D1, D2).  Returns 1 if the request goes to the network, else
+// writes the local / dropped / failed code to `code`.
+__device__ __forceinline__ bool origin_offloads(const Net& n, uint32_t r, uint32_t o, const Rnd4& rx, int& code)
+{
+    if (o >= n.N) { set_error(n, eArg, o); code = -3; return false; }
+    const size_t ox = size_t(r) * n.N + o;
+    if (!n.online[ox]) { code = -3; return false; }
+    const uint32_t cap = n.cap_eff[ox];
+    code = cap == 0 ? -4 : -1;
+    return util_at_least(cap, n.backlog[ox], n.util_window_ms, n.offload_util_pm[ox]) &&
+           ppm(rx.w[0]) < n.offload_ppm[ox] && n.credit[ox] >= n.R;
+}
+
+// ---- settlement of one request (one thread) ----------------------------------------------------
+
+__device__ __forceinline__ void add64(long long* p, long long v) { atomicAdd((unsigned long long*)p, (unsigned long long)v); }
+
+struct SettleAcc {
+    uint32_t c[sSumLat];           // counters before sSumLat are small
+    unsigned long long sum_lat;
+};
+
+__device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t o, uint32_t li, uint32_t lo, int a, int b,
+                                           const int (&jd)[4], uint32_t oc, bool near, SettleAcc& s)
+{
+    const size_t base = size_t(r) * n.N;
+    const uint64_t work = uint64_t(li) + lo;
+    s.c[sRequests]++;
+    if (near) s.c[sNear]++;
+    if (a == -3) { s.c[sDropped]++; return; }
+    if (a == -4) { s.c[sFailed]++; return; }
+    uint32_t ex;
+    if (a < 0) {
+        s.c[a == -1 ? sLocal : sFallback]++;
+        add64(&n.d_backlog[base + o], (long long)work);
+        atomicAdd(&n.served_local[base + o], 1ull);
+        ex = o;
+    } else {
+        s.c[sDelegated]++;
+        long long pay = n.R;
+        add64(&n.d_credit[base + a], n.R);
+        add64(&n.d_backlog[base + a], (long long)work);
+        atomicAdd(&n.served[base + a], 1ull);
+        ex = uint32_t(a);
+        if (oc != 0) s.c[sDuel]++;
+        if (oc == 4) s.c[sDuelCancelled]++;
+        if (oc >= 1 && oc <= 3) {
+            pay += n.R;
+            add64(&n.d_credit[base + b], n.R);
+            add64(&n.d_backlog[base + b], (long long)work);
+            atomicAdd(&n.served[base + b], 1ull);
+            atomicAdd(&n.d_duels[base + a], 1u);
+            atomicAdd(&n.d_duels[base + b], 1u);
+            int nj = 0;
+#pragma unroll
+            for (int l = 0; l < 4; ++l)
+                if (jd[l] >= 0) { add64(&n.d_backlog[base + jd[l]], (long long)(uint64_t(li) + 2ull * lo)); ++nj; }
+            s.c[sJudgeEvals] += nj;
+            if (oc == 3) s.c[sDraw]++;
+            else {
+                const int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
+                const long long pot = n.P - n.R_add, share = pot / nj;
+                add64(&n.d_credit[base + lose], -n.P);
+                add64(&n.d_credit[base + win], n.R_add + (pot - share * nj));
+                atomicAdd(&n.d_wins[base + win], 1u);
+#pragma unroll
+                for (int l = 0; l < 4; ++l)
+                    if (jd[l] >= 0) add64(&n.d_credit[base + jd[l]], share);
+            }
+        }
+        add64(&n.d_credit[base + o], -pay);
+    }
+    const uint64_t cap = n.cap_eff[base + ex];
+    const uint64_t t = (uint64_t(n.backlog[base + ex]) + work) * 1000ull, tq = t / cap;
+    const uint64_t lat = tq + (tq * cap != t ? 1 : 0) + (a >= 0 ? n.hop_ms : 0);
+    const uint64_t ideal = (work * 1000ull + n.cap_ref - 1) / n.cap_ref;
+    const uint64_t deadline = uint64_t(n.slo_num) * ideal / n.slo_den;
+    s.sum_lat += lat;
+    if (lat <= deadline) s.c[sSloMet]++;
+}
+
+__device__ __forceinline__ void acc_zero(SettleAcc& s)
+{
+#pragma unroll
+    for (int k = 0; k < int(sSumLat); ++k) s.c[k] = 0;
+    s.sum_lat = 0;
+}
+__device__ __forceinline__ void acc_flush(BlockStats& bs, const SettleAcc& s)
+{
+#pragma unroll
+    for (int k = 0; k < int(sSumLat); ++k) stats_add(bs, k, s.c[k]);
+    stats_add(bs, sSumLat, s.sum_lat);
+}
+
+}  // namespace wwws
