@@ -51,6 +51,9 @@ typedef enum {
 #define WWWS_MAX_JUDGES 4u
 #define WWWS_FLAG_REPUTATION 1u /* multiply the PoS weight by the smoothed duel win rate */
 #define WWWS_FLAG_LOAD 2u       /* multiply the PoS weight by the advertised spare-capacity fraction */
+#define WWWS_FLAG_GREEDY 4u     /* customised rule: instead of drawing in proportion to the weights, take the
+                                   candidate with the highest weight (lowest id on ties), then the next one on
+                                   refusal; flags bit 0 then marks a runner-up within 1e-5 (relative) of the pick */
 
 /* Plain data, copied at creation.  Probabilities are in parts per million. */
 typedef struct {
@@ -124,6 +127,10 @@ typedef struct {
     uint64_t n_requests, n_local, n_fallback_local, n_dropped, n_failed, n_delegated, n_duel, n_duel_cancelled,
         n_draw, n_judge_evals, n_probes, n_near_boundary, slo_met, sum_latency_ms, n_offline_marks, rounds, blocks;
     int64_t credit_total; /* finalized + pending credit of all peers */
+    uint64_t chain_head;     /* id of the last finalized credit block (Table "Structure of a Credit Block"):
+                                hash of the parent id, the block's operations digest and its height */
+    uint64_t pending_digest; /* order-independent digest (wrapping sum of per-record hashes) of the credit
+                                operations settled since the last finalization */
 } wwws_stats_t;
 
 /* Per-peer tables for wwws_export_table / wwws_import_table; element type in the comment. */

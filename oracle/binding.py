@@ -19,7 +19,7 @@ _SO = os.path.join(_HERE, "libwwws_oracle.so")
 
 STAT_NAMES = ("n_requests", "n_local", "n_fallback_local", "n_dropped", "n_failed", "n_delegated", "n_duel",
               "n_duel_cancelled", "n_draw", "n_judge_evals", "n_probes", "n_near_boundary", "slo_met",
-              "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total")
+              "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest")
 TABLES = ("online", "cap_eff", "backlog", "ver", "credit", "stake", "wins", "duels", "served", "served_local",
           "d_credit", "d_wins", "d_duels")
 
@@ -79,6 +79,7 @@ def lib():
         L.orc_below.restype = C.c_uint32; L.orc_below.argtypes = [C.c_uint32, C.c_uint32]
         L.orc_mulhi64.restype = C.c_uint64; L.orc_mulhi64.argtypes = [C.c_uint64, C.c_uint64]
         L.orc_merge.restype = C.c_uint64; L.orc_merge.argtypes = [C.c_uint64, C.c_uint64]
+        L.orc_mix64.restype = C.c_uint64; L.orc_mix64.argtypes = [C.c_uint64]
         for name, ct in (("orc_view", C.c_uint64), ("orc_exec_a", C.c_int32), ("orc_exec_b", C.c_int32),
                          ("orc_judges", C.c_int32), ("orc_outcome", C.c_uint8), ("orc_flags", C.c_uint8),
                          ("orc_score_a", C.c_float), ("orc_score_sum", C.c_float)):
@@ -171,7 +172,7 @@ class Oracle:
     def stats_dict(self, row=-1):
         s = self.stats()[row]
         d = {k: int(v) for k, v in zip(STAT_NAMES, s)}
-        d["credit_total"] = int(np.int64(s[len(STAT_NAMES) - 1]))
+        d["credit_total"] = int(np.int64(s[STAT_NAMES.index("credit_total")]))
         return d
 
     def table(self, name):

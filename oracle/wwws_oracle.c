@@ -112,7 +112,8 @@ typedef struct {
 } peer_t;
 
 enum { S_REQUESTS, S_LOCAL, S_FALLBACK, S_DROPPED, S_FAILED, S_DELEGATED, S_DUEL, S_DUEL_CANCELLED, S_DRAW,
-       S_JUDGE_EVALS, S_PROBES, S_NEAR, S_SLO_MET, S_SUM_LAT, S_OFFLINE_MARKS, S_ROUNDS, S_BLOCKS, S_CREDIT_TOTAL, S_N };
+       S_JUDGE_EVALS, S_PROBES, S_NEAR, S_SLO_MET, S_SUM_LAT, S_OFFLINE_MARKS, S_ROUNDS, S_BLOCKS, S_CREDIT_TOTAL,
+       S_CHAIN_HEAD, S_PENDING_DIGEST, S_N };
 
 typedef struct {
     uint32_t inplay;       /* lanes still in play after the draws so far */
@@ -169,6 +170,30 @@ static uint32_t cap_eff_at(const orc_net *n, const peer_t *p, uint32_t j, uint32
 
 static uint64_t adv_cap_of(const peer_t *p) { return (uint64_t)p->cap_eff * p->misreport_mul; }
 
+/* Credit Block Chain (Table "Structure of a Credit Block"): a block holds a list of credit
+ * operations, its own id and its parent's id.  Here a block's operations are summarised by an
+ * order-independent 64-bit digest (the wrapping sum of one hash per ledger record), and the block
+ * id chains that digest to the parent id.  The mixer is the SplitMix64 finaliser (Steele, Lea,
+ * Flood 2014); it stands in for the cryptographic hash, signatures are out of scope. */
+#define GAMMA 0x9E3779B97F4A7C15ULL
+uint64_t orc_mix64(uint64_t z)
+{
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
+    z ^= z >> 27; z *= 0x94D049BB133111EBULL;
+    z ^= z >> 31;
+    return z;
+}
+static uint64_t chain_key(const orc_net *n, uint32_t r) { return n->cfg.seed ^ ((uint64_t)(r + n->cfg.replica_offset) * GAMMA); }
+
+/* one ledger record: request q moves `amount` credits on `peer`'s account; kind says why */
+enum { OP_PAY = 1, OP_EARN = 2, OP_PAY_CHALLENGER = 3, OP_EARN_CHALLENGER = 4, OP_PENALTY = 5, OP_REWARD = 6, OP_JUDGE = 7 };
+static void post(orc_net *n, uint32_t r, uint32_t q, uint32_t kind, uint32_t peer, int64_t amount)
+{
+    n->peers[(size_t)r * n->N + peer].d_credit += amount;
+    uint64_t word = ((uint64_t)q << 32) | ((uint64_t)kind << 24) | peer;
+    n->stats[(size_t)r * S_N + S_PENDING_DIGEST] += orc_mix64(orc_mix64(chain_key(n, r) ^ word) + (uint64_t)amount);
+}
+
 /* S5 finalize = commit of a credit block (Section "Credit-based Transaction System"):
  * pending operations are folded into the ledger, stake is re-derived, total credit is checked. */
 static void finalize_replica(orc_net *n, uint32_t r)
@@ -182,7 +207,10 @@ static void finalize_replica(orc_net *n, uint32_t r)
         p->stake = pos * p->stake_pm / 1000;
         total += p->credit;
     }
-    n->stats[(size_t)r * S_N + S_BLOCKS] += 1;
+    uint64_t *st = &n->stats[(size_t)r * S_N];
+    st[S_BLOCKS] += 1;
+    st[S_CHAIN_HEAD] = orc_mix64(orc_mix64(st[S_CHAIN_HEAD] ^ chain_key(n, r)) + st[S_PENDING_DIGEST] + GAMMA * st[S_BLOCKS]);
+    st[S_PENDING_DIGEST] = 0;
     if (total != n->credit_total0[r]) n->error = 6;
 }
 
@@ -223,6 +251,7 @@ orc_net *orc_create(const orc_config *cfg, const orc_peer_init *in)
         }
         finalize_replica(n, r);
         n->stats[(size_t)r * S_N + S_BLOCKS] = 0;
+        n->stats[(size_t)r * S_N + S_CHAIN_HEAD] = orc_mix64(chain_key(n, r));      /* genesis id */
         /* every node starts knowing every peer, possibly by a version a few rounds old */
         for (uint32_t i = 0; i < n->N; ++i)
             for (uint32_t j = 0; j < n->N; ++j) {
@@ -403,6 +432,20 @@ static pick_t pos_draw(const orc_net *n, uint32_t rg, uint32_t q, const window_t
     for (int c = 0; c < WIN; ++c) if (ct->inplay >> c & 1) S += w->W[c];
     if (S == 0) return out;
     uint32_t d = ct->n_draws++;
+    if (n->cfg.flags & 4) {
+        /* greedy rule (a customised load-balancing rule of the Policy Manager): the highest
+         * weight wins, the lowest lane on ties; flagged when the runner-up is within 1e-5 */
+        int best = -1, second = -1;
+        for (int c = 0; c < WIN; ++c) {
+            if (!(ct->inplay >> c & 1) || w->W[c] == 0) continue;
+            if (best < 0 || w->W[c] > w->W[best]) { second = best; best = c; }
+            else if (second < 0 || w->W[c] > w->W[second]) second = c;
+        }
+        out.lane = best;
+        out.near = second >= 0 && w->W[best] - w->W[second] <= w->W[best] / 100000;
+        ct->inplay &= ~(1u << best);
+        return out;
+    }
     rnd4 y = draw(n->cfg.seed, q, d / 2, rg, ST_DRAW, 0);
     uint64_t u = ((uint64_t)y.w[2 * (d % 2)] << 32) | y.w[2 * (d % 2) + 1];
     uint64_t r64 = orc_mulhi64(u, S), acc = 0;
@@ -550,14 +593,14 @@ int orc_settle_credits(orc_net *n, int finalize)
                 P[o].d_backlog += (int64_t)work; P[o].served_local += 1; ex = o;
             } else {                                                         /* S2 credits-for-offloading */
                 st[S_DELEGATED] += 1;
-                P[o].d_credit -= c->reward_R; P[a].d_credit += c->reward_R;
+                post(n, r, (uint32_t)q, OP_PAY, o, -c->reward_R); post(n, r, (uint32_t)q, OP_EARN, (uint32_t)a, c->reward_R);
                 P[a].d_backlog += (int64_t)work; P[a].served += 1; ex = (uint32_t)a;
                 uint8_t oc = n->outcome[x];
                 if (oc != 0) st[S_DUEL] += 1;
                 if (oc == 4) st[S_DUEL_CANCELLED] += 1;
                 if (oc >= 1 && oc <= 3) {                                    /* S3 duel */
                     int b = n->exec_b[x], nj = 0;
-                    P[o].d_credit -= c->reward_R; P[b].d_credit += c->reward_R;
+                    post(n, r, (uint32_t)q, OP_PAY_CHALLENGER, o, -c->reward_R); post(n, r, (uint32_t)q, OP_EARN_CHALLENGER, (uint32_t)b, c->reward_R);
                     P[b].d_backlog += (int64_t)work; P[b].served += 1;
                     P[a].d_duels += 1; P[b].d_duels += 1;
                     for (int l = 0; l < 4; ++l) if (n->judges[4 * x + l] >= 0) {
@@ -568,10 +611,10 @@ int orc_settle_credits(orc_net *n, int finalize)
                     else {
                         int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
                         int64_t pot = c->penalty_P - c->reward_add, share = pot / nj;
-                        P[lose].d_credit -= c->penalty_P;
-                        P[win].d_credit += c->reward_add + (pot - share * nj);
+                        post(n, r, (uint32_t)q, OP_PENALTY, (uint32_t)lose, -c->penalty_P);
+                        post(n, r, (uint32_t)q, OP_REWARD, (uint32_t)win, c->reward_add + (pot - share * nj));
                         P[win].d_wins += 1;
-                        for (int l = 0; l < 4; ++l) if (n->judges[4 * x + l] >= 0) P[n->judges[4 * x + l]].d_credit += share;
+                        for (int l = 0; l < 4; ++l) if (n->judges[4 * x + l] >= 0) post(n, r, (uint32_t)q, OP_JUDGE + (uint32_t)l, (uint32_t)n->judges[4 * x + l], share);
                     }
                 }
             }

@@ -190,6 +190,7 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
     d.prio_window_ms = cfg->prio_window_ms; d.util_window_ms = cfg->util_window_ms; d.cap_ref = cfg->cap_ref_tok_s;
     d.slo_num = cfg->slo_num; d.slo_den = cfg->slo_den; d.hop_ms = cfg->hop_ms; d.flags = cfg->flags; d.n_rank = cfg->n_rank;
     d.R = cfg->reward_R; d.R_add = cfg->reward_add; d.P = cfg->penalty_P;
+    for (int k = 0; k < 4; ++k) d.judge_share[k] = (d.P - d.R_add) / (k + 1);
     d.uwf = float(cfg->util_window_ms) / 1000.0f;
     d.max_batch = cfg->max_batch;
 
@@ -215,7 +216,12 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
     for (uint32_t r = 0; r < d.Rp; ++r)
         for (uint32_t j = 0; j < d.N; ++j) tot[r] += init->credit0[size_t(r) * d.N + j];
     CUDA_TRY(nullptr, cudaMemcpyAsync(const_cast<int64_t*>(d.credit_total0), tot.data(), d.Rp * 8ull, cudaMemcpyHostToDevice, s));
-    CUDA_TRY(nullptr, cudaMemsetAsync(d.stats, 0, uint64_t(d.Rp) * sCount * 8, s));
+    {   // counters start at zero, each replica's chain at its genesis id
+        std::vector<unsigned long long> st0(size_t(d.Rp) * sCount, 0);
+        for (uint32_t r = 0; r < d.Rp; ++r)
+            st0[size_t(r) * sCount + sChainHead] = mix64(cfg->seed ^ (uint64_t(r + cfg->replica_offset) * kGamma));
+        CUDA_TRY(nullptr, cudaMemcpy(d.stats, st0.data(), st0.size() * 8, cudaMemcpyHostToDevice));
+    }
     CUDA_TRY(nullptr, cudaMemsetAsync(d.credit_check, 0, d.Rp * 8ull, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.err, 0, 16, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.partner, 0xff, NP * 16, s));

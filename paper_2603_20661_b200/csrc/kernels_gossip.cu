@@ -55,9 +55,9 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
 // streaming (evict-first) so that they do not push the panel out.
 //
 // A thread moves 32 bytes (four entries) per row it touches: one 256-bit load per source row.
-constexpr int kMergeThreads = 256;
+
+constexpr int kMergeThreads = 128;
 constexpr int kMergeIters = 4;                         // rows per thread
-constexpr int kMergeMaxRows = 128;                     // rows per block at the narrowest panel
 
 struct Q4 { uint64_t a, b, c, d; };                    // four entries = 32 bytes
 
@@ -82,10 +82,10 @@ __device__ __forceinline__ void join(Q4& x, const Q4& y)
 // panel and walks kMergeIters rows of the block's row group.  Prologue: every row of the group
 // resolves its sources once (partner rows that answered, -1 otherwise) into shared memory, so
 // the streaming part has no dependent metadata loads.
-__global__ void __launch_bounds__(kMergeThreads, 4) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
+__global__ void __launch_bounds__(kMergeThreads, 8) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
                                                                      uint32_t n_panels, uint32_t groups_per_panel)
 {
-    __shared__ int4 s_src[kMergeMaxRows];
+    __shared__ int4 s_src[kMergeThreads / 8 * kMergeIters];
     const uint32_t b = blockIdx.x;
     const uint32_t per_replica = n_panels * groups_per_panel;
     const uint32_t r = b / per_replica;
@@ -160,7 +160,7 @@ __global__ void k_gossip_fixup(Net n)
     if (marks) atomicAdd(&n.stats[size_t(r) * sCount + sOfflineMarks], (unsigned long long)marks);
 }
 
-// Panel width: the widest power of two (32 .. 1024 columns) whose panel of N rows fits the
+// Panel width: the widest power of two (32 .. 512 columns) whose panel of N rows fits the
 // L2 budget; WWWS_PANEL_BYTES overrides the budget (tuning).
 static uint32_t panel_columns(const Net& n)
 {
@@ -169,7 +169,7 @@ static uint32_t panel_columns(const Net& n)
         const uint64_t v = e ? strtoull(e, nullptr, 10) : 0;
         return v ? v : (16ull << 20);
     }();
-    uint32_t pc = 1024;
+    uint32_t pc = 4 * kMergeThreads;                                      // one pass of the block covers at least one row segment
     while (pc > 32 && uint64_t(n.N) * pc * 8 > budget) pc >>= 1;
     return pc;
 }

@@ -99,7 +99,11 @@ __global__ void k_finalize_check(Net n)
     if (r >= n.Rp) return;
     if (n.credit_check[r] != n.credit_total0[r]) set_error(n, eInvariant, r);
     n.credit_check[r] = 0;
-    n.stats[size_t(r) * sCount + sBlocks] += 1;
+    unsigned long long* st = n.stats + size_t(r) * sCount;
+    st[sBlocks] += 1;
+    // block id = hash of (parent id, order-independent digest of the block's records, height)
+    st[sChainHead] = mix64(mix64(st[sChainHead] ^ chain_key(n, r)) + st[sPendingDigest] + kGamma * st[sBlocks]);
+    st[sPendingDigest] = 0;
 }
 
 // Re-derive stake and weight from the ledger as it stands (after a table import).

@@ -44,6 +44,19 @@ __device__ __forceinline__ int pos_draw(const Net& n, Window& w, uint32_t lane)
     const uint64_t S = __shfl_sync(kFull, incl, 31);
     if (S == 0) return -1;
     const uint32_t d = w.n_draws++;
+    if (n.flags & 4u) {
+        // greedy rule: highest weight, lowest lane on ties; flagged when the runner-up is within 1e-5
+        uint64_t m = w.W;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) { const uint64_t t = __shfl_xor_sync(kFull, m, o); m = t > m ? t : m; }
+        const int pick = __ffs(__ballot_sync(kFull, w.W == m)) - 1;
+        uint64_t m2 = lane == uint32_t(pick) ? 0 : w.W;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) { const uint64_t t = __shfl_xor_sync(kFull, m2, o); m2 = t > m2 ? t : m2; }
+        if (m2 != 0 && m - m2 <= m / 100000ull) w.near = true;
+        if (lane == uint32_t(pick)) w.W = 0;
+        return pick;
+    }
     if (w.y_slot != (d >> 1)) { w.y = draw(n, w.q, d >> 1, w.rg, kDraw); w.y_slot = d >> 1; }
     const uint64_t u = (d & 1u) ? (uint64_t(w.y.w[2]) << 32 | w.y.w[3]) : (uint64_t(w.y.w[0]) << 32 | w.y.w[1]);
     const uint64_t r64 = __umul64hi(u, S);
@@ -196,7 +209,7 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
         const size_t x = size_t(r) * n.Q + first + idx;
         const int4 j4 = *reinterpret_cast<const int4*>(n.judges + 4 * x);
         const int jd[4] = { j4.x, j4.y, j4.z, j4.w };
-        settle_one(n, r, n.origin[x], n.len_in[x], n.len_out[x], n.exec_a[x], n.exec_b[x], jd, n.outcome[x],
+        settle_one(n, r, uint32_t(first + idx), n.origin[x], n.len_in[x], n.len_out[x], n.exec_a[x], n.exec_b[x], jd, n.outcome[x],
                    (n.rflags[x] & 1) != 0, s);
     }
 #pragma unroll
@@ -207,6 +220,9 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
     unsigned long long sl = s.sum_lat;
     for (int o = 16; o; o >>= 1) sl += __shfl_down_sync(kFull, sl, o);
     if ((threadIdx.x & 31) == 0) stats_add(bs, sSumLat, sl);
+    unsigned long long dg = s.digest;
+    for (int o = 16; o; o >>= 1) dg += __shfl_down_sync(kFull, dg, o);
+    if ((threadIdx.x & 31) == 0) stats_add(bs, sPendingDigest, dg);
     stats_end(n, bs, r);
 }
 

@@ -39,6 +39,22 @@ __device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, 
     const uint64_t S = d.G0 + d.G1 + d.G2 + d.G3;
     if (S == 0) return -1;
     const uint32_t k = d.n_draws++;
+    if (n.flags & 4u) {
+        // greedy rule: highest weight, lowest lane on ties; flagged when the runner-up is within 1e-5
+        uint64_t m = 0, m2 = 0;
+        int pick = -1;
+#pragma unroll 8
+        for (int c = 0; c < int(kWin); ++c) {
+            const uint64_t w = sh.W[c][slot];
+            if (w > m) { m2 = m; m = w; pick = c; }
+            else if (w > m2) m2 = w;
+        }
+        if (m2 != 0 && m - m2 <= m / 100000ull) d.near = true;
+        sh.W[pick][slot] = 0;
+        const int g = pick >> 3;
+        if (g == 0) d.G0 -= m; else if (g == 1) d.G1 -= m; else if (g == 2) d.G2 -= m; else d.G3 -= m;
+        return pick;
+    }
     if (d.y_slot != (k >> 1)) { d.y = draw(n, q, k >> 1, rg, kDraw); d.y_slot = k >> 1; }
     const uint64_t u = (k & 1u) ? (uint64_t(d.y.w[2]) << 32 | d.y.w[3]) : (uint64_t(d.y.w[0]) << 32 | d.y.w[1]);
     const uint64_t r64 = __umul64hi(u, S);
@@ -160,7 +176,7 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
             *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(-1, -1, -1, -1);
             const int jd[4] = { -1, -1, -1, -1 };
             acc.c[sProbes] += d.n_probes;
-            settle_one(n, r, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
+            settle_one(n, r, q, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
         }
     }
     __syncthreads();
@@ -213,7 +229,7 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
         n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = d.near ? 1 : 0;
         *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
         acc.c[sProbes] += d.n_probes;
-        settle_one(n, r, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
+        settle_one(n, r, q, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
     }
 
     // ---- counters: warp reduce, block reduce, one atomic per counter and block ---------------
@@ -225,6 +241,9 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
     unsigned long long sl = acc.sum_lat;
     for (int o = 16; o; o >>= 1) sl += __shfl_down_sync(kFull, sl, o);
     if ((threadIdx.x & 31) == 0) stats_add(sh.stats, sSumLat, sl);
+    unsigned long long dg = acc.digest;
+    for (int o = 16; o; o >>= 1) dg += __shfl_down_sync(kFull, dg, o);
+    if ((threadIdx.x & 31) == 0) stats_add(sh.stats, sPendingDigest, dg);
     stats_end(n, sh.stats, r);
 }
 

@@ -84,6 +84,13 @@ __device__ __forceinline__ bool origin_offloads(const Net& n, uint32_t r, uint32
            ppm(rx.w[0]) < n.offload_ppm[ox] && n.credit[ox] >= n.R;
 }
 
+// 64-bit by 32-bit unsigned division; the common case (numerator below 2^32) takes the short
+// 32-bit path instead of the long emulated 64-bit one.
+__device__ __forceinline__ uint64_t udiv64by32(uint64_t t, uint32_t d)
+{
+    return (t >> 32) == 0 ? uint64_t(uint32_t(t) / d) : t / d;
+}
+
 // ---- settlement of one request (one thread) ----------------------------------------------------
 
 __device__ __forceinline__ void add64(long long* p, long long v) { atomicAdd((unsigned long long*)p, (unsigned long long)v); }
@@ -91,9 +98,10 @@ __device__ __forceinline__ void add64(long long* p, long long v) { atomicAdd((un
 struct SettleAcc {
     uint32_t c[sSumLat];           // counters before sSumLat are small
     unsigned long long sum_lat;
+    unsigned long long digest;     // wrapping sum of the record hashes of this thread's requests
 };
 
-__device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t o, uint32_t li, uint32_t lo, int a, int b,
+__device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q, uint32_t o, uint32_t li, uint32_t lo, int a, int b,
                                            const int (&jd)[4], uint32_t oc, bool near, SettleAcc& s)
 {
     const size_t base = size_t(r) * n.N;
@@ -110,7 +118,9 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t o,
         ex = o;
     } else {
         s.c[sDelegated]++;
+        const uint64_t key = chain_key(n, r);
         long long pay = n.R;
+        s.digest += record_hash(key, q, opPay, o, -n.R) + record_hash(key, q, opEarn, uint32_t(a), n.R);
         add64(&n.d_credit[base + a], n.R);
         add64(&n.d_backlog[base + a], (long long)work);
         atomicAdd(&n.served[base + a], 1ull);
@@ -119,6 +129,7 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t o,
         if (oc == 4) s.c[sDuelCancelled]++;
         if (oc >= 1 && oc <= 3) {
             pay += n.R;
+            s.digest += record_hash(key, q, opPayChallenger, o, -n.R) + record_hash(key, q, opEarnChallenger, uint32_t(b), n.R);
             add64(&n.d_credit[base + b], n.R);
             add64(&n.d_backlog[base + b], (long long)work);
             atomicAdd(&n.served[base + b], 1ull);
@@ -132,22 +143,27 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t o,
             if (oc == 3) s.c[sDraw]++;
             else {
                 const int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
-                const long long pot = n.P - n.R_add, share = pot / nj;
+                const long long pot = n.P - n.R_add, share = n.judge_share[nj - 1];
+                const long long prize = n.R_add + (pot - share * nj);
+                s.digest += record_hash(key, q, opPenalty, uint32_t(lose), -n.P) + record_hash(key, q, opReward, uint32_t(win), prize);
                 add64(&n.d_credit[base + lose], -n.P);
-                add64(&n.d_credit[base + win], n.R_add + (pot - share * nj));
+                add64(&n.d_credit[base + win], prize);
                 atomicAdd(&n.d_wins[base + win], 1u);
 #pragma unroll
                 for (int l = 0; l < 4; ++l)
-                    if (jd[l] >= 0) add64(&n.d_credit[base + jd[l]], share);
+                    if (jd[l] >= 0) {
+                        s.digest += record_hash(key, q, opJudge + l, uint32_t(jd[l]), share);
+                        add64(&n.d_credit[base + jd[l]], share);
+                    }
             }
         }
         add64(&n.d_credit[base + o], -pay);
     }
     const uint64_t cap = n.cap_eff[base + ex];
-    const uint64_t t = (uint64_t(n.backlog[base + ex]) + work) * 1000ull, tq = t / cap;
+    const uint64_t t = (uint64_t(n.backlog[base + ex]) + work) * 1000ull, tq = udiv64by32(t, uint32_t(cap));
     const uint64_t lat = tq + (tq * cap != t ? 1 : 0) + (a >= 0 ? n.hop_ms : 0);
-    const uint64_t ideal = (work * 1000ull + n.cap_ref - 1) / n.cap_ref;
-    const uint64_t deadline = uint64_t(n.slo_num) * ideal / n.slo_den;
+    const uint64_t ideal = udiv64by32(work * 1000ull + n.cap_ref - 1, n.cap_ref);
+    const uint64_t deadline = udiv64by32(uint64_t(n.slo_num) * ideal, n.slo_den);
     s.sum_lat += lat;
     if (lat <= deadline) s.c[sSloMet]++;
 }
@@ -157,12 +173,14 @@ __device__ __forceinline__ void acc_zero(SettleAcc& s)
 #pragma unroll
     for (int k = 0; k < int(sSumLat); ++k) s.c[k] = 0;
     s.sum_lat = 0;
+    s.digest = 0;
 }
 __device__ __forceinline__ void acc_flush(BlockStats& bs, const SettleAcc& s)
 {
 #pragma unroll
     for (int k = 0; k < int(sSumLat); ++k) stats_add(bs, k, s.c[k]);
     stats_add(bs, sSumLat, s.sum_lat);
+    stats_add(bs, sPendingDigest, s.digest);
 }
 
 }  // namespace wwws

@@ -15,7 +15,8 @@ enum : uint32_t { kOrigin = 1, kDraw = 2, kProbe = 3, kJudge = 4, kGossip = 5, k
 
 // Per-replica counters, in the order of wwws_stats_t.
 enum : uint32_t { sRequests, sLocal, sFallback, sDropped, sFailed, sDelegated, sDuel, sDuelCancelled, sDraw,
-                  sJudgeEvals, sProbes, sNear, sSloMet, sSumLat, sOfflineMarks, sRounds, sBlocks, sCreditTotal, sCount };
+                  sJudgeEvals, sProbes, sNear, sSloMet, sSumLat, sOfflineMarks, sRounds, sBlocks, sCreditTotal,
+                  sChainHead, sPendingDigest, sCount };
 
 // Device error word codes (subset of wwws_status).
 enum : uint32_t { eArg = 1, eRange = 4, eInvariant = 6 };
@@ -30,6 +31,7 @@ struct Net {
     uint32_t p_duel, p_noise, p_leave, p_join, p_prio;
     uint32_t prio_window_ms, util_window_ms, cap_ref, slo_num, slo_den, hop_ms, flags, n_rank;
     int64_t R, R_add, P;
+    int64_t judge_share[4];                      // (P - R_add) / n for n = 1..4 judges
     float uwf;                                   // util_window_ms / 1000 in fp32
     // view double buffer
     uint64_t* view; uint64_t* view_new;
@@ -108,6 +110,26 @@ __device__ __forceinline__ uint32_t cap_eff_at(const Net& n, uint32_t cap_true, 
     if (!prio) return cap_true;
     const uint32_t w = now_ms / n.prio_window_ms;
     return ppm(draw(n, j, w, rg, kPrio).w[0]) < n.p_prio ? cap_true / 2 : cap_true;
+}
+
+// Credit block chain: SplitMix64 finaliser (Steele, Lea, Flood 2014) as the record and block hash.
+constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27; z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
+}
+__device__ __forceinline__ uint64_t chain_key(const Net& n, uint32_t r)
+{
+    return (uint64_t(n.key1) << 32 | n.key0) ^ (uint64_t(r + n.replica_offset) * kGamma);
+}
+// Hash of one ledger record: request q moves `amount` credits on `peer`'s account, for reason `kind`.
+enum : uint32_t { opPay = 1, opEarn = 2, opPayChallenger = 3, opEarnChallenger = 4, opPenalty = 5, opReward = 6, opJudge = 7 };
+__device__ __forceinline__ uint64_t record_hash(uint64_t key, uint32_t q, uint32_t kind, uint32_t peer, int64_t amount)
+{
+    return mix64(mix64(key ^ (uint64_t(q) << 32 | uint64_t(kind) << 24 | peer)) + uint64_t(amount));
 }
 
 __device__ __forceinline__ void set_error(const Net& n, uint32_t code, uint32_t detail)

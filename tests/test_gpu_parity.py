@@ -155,6 +155,9 @@ def test_edge_cases_match_oracle():
                           p_noise_ppm=500_000, hop_ms=25, flags=0, p_leave_ppm=200_000, p_join_ppm=500_000,
                           peers={"stake_pm": rng.integers(0, 1001, 64), "credit0": rng.integers(0, 300, 64),
                                  "prio_flag": 1, "misreport_mul": rng.integers(1, 5, 64)}))
+    # greedy rule, with ties (equal stakes) and refusals
+    cases.append(make_net(70, n_requests=400, seed=9, origin=rng.integers(0, 70, 400), flags=3 | 4, p_duel_ppm=400_000,
+                          peers={"accept_ppm": 600_000, "stake_pm": rng.integers(1, 4, 70) * 300}))
     for ci, (st, pa, rq) in enumerate(cases):
         g = Network(st, pa, 128); g.bind_requests(rq)
         o = Oracle(st, pa); o.bind_requests(rq)

@@ -259,3 +259,54 @@ def test_truly_offline_peers_never_serve_or_judge():
     assert decided.mean() > 0.9
     assert np.all((res["judges"][0][decided] >= 0).sum(-1) == 3)     # 7 live candidates: always a full panel
     assert o.stats_dict()["n_probes"] > 2 * Q                          # refused probes were spent on the dead
+
+
+def test_greedy_rule_takes_the_best_weight_then_the_next():
+    """Greedy dispatch (flag 4): executor = highest weight of the window recomputed by the
+    second routine; a refusing best candidate hands over to the runner-up; ties go to the
+    lowest id; the flag marks a runner-up within 1e-5."""
+    N, Q = 70, 1500
+    rng = np.random.default_rng(3)
+    peers = {"cap_true_tok_s": rng.integers(500, 8000, N), "stake_pm": rng.integers(1, 1001, N)}
+    st, pa, rq = make_net(N, n_requests=Q, seed=9, flags=3 | 4, p_duel_ppm=1_000_000, n_judges=2, peers=peers,
+                          origin=rng.integers(0, N, Q), max_probes=2)
+    o = Oracle(st, pa); o.bind_requests(rq)
+    for s in range(2):
+        o.run_step(s * 500, 500, 1000 * (s + 1), True)
+    o.advance_time(3000); o.gossip_round()
+    view = o.view()[0]; stake = o.table("stake")[0]; wins = o.table("wins")[0]; duels = o.table("duels")[0]
+    o.dispatch_batch(1000, 500); o.duel_judge()
+    res = o.results()
+    n_chk = 0
+    for q in range(1000, 1500):
+        a = res["exec_a"][0, q]
+        if a < 0:
+            continue
+        orig = int(rq["origin"][0, q])
+        _, _, blk = o.window_weights(0, q)
+        W, _ = _weights_second_routine(st, view[orig], stake, wins, duels, orig, blk)
+        order = sorted(range(32), key=lambda c: (-int(W[c]), c))
+        order = [c for c in order if W[c] > 0]
+        got = [a, res["exec_b"][0, q]] + list(res["judges"][0, q, :2])
+        got = [g - 32 * blk for g in got if g >= 0]
+        assert got == order[:len(got)], (q, got, order[:6])     # all peers accept: strict weight order
+        n_chk += 1
+    assert n_chk > 300
+    # refusal: the best candidate never accepts -> the runner-up serves; tie -> lowest id
+    st2, pa2, rq2 = make_net(6, n_requests=50, flags=4, p_duel_ppm=0,
+                             peers=requester_first(6, credit0=np.array([10 ** 6, 500, 900, 900, 100, 100]),
+                                                   accept_ppm=np.array([0, 10 ** 6, 0, 10 ** 6, 10 ** 6, 10 ** 6])))
+    o2 = Oracle(st2, pa2); o2.bind_requests(rq2)
+    o2.dispatch_batch(0, 50)
+    r2 = o2.results()
+    assert np.all(r2["exec_a"][0] == 3)           # 2 and 3 tie at the top, 2 is asked first and refuses
+    assert np.all(r2["flags"][0] & 1 == 1)        # a tie is as near as it gets
+    assert o2.stats_dict()["n_probes"] == 100
+    # near flag threshold: weights 256*100000 vs 256*99999 differ by 256 <= W/100000 = 256 -> flagged;
+    # 256*100000 vs 256*99998 differ by 512 -> not flagged
+    for other, flagged in ((99_999, 1), (99_998, 0)):
+        st3, pa3, rq3 = make_net(3, n_requests=4, flags=4, p_duel_ppm=0,
+                                 peers=requester_first(3, credit0=np.array([10 ** 6, 100_000, other])))
+        o3 = Oracle(st3, pa3); o3.bind_requests(rq3)
+        o3.dispatch_batch(0, 4)
+        assert np.all(o3.results()["exec_a"][0] == 1) and np.all((o3.results()["flags"][0] & 1) == flagged)
