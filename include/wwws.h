@@ -51,6 +51,8 @@ typedef enum {
 #define WWWS_MAX_JUDGES 4u
 #define WWWS_FLAG_REPUTATION 1u /* multiply the PoS weight by the smoothed duel win rate */
 #define WWWS_FLAG_LOAD 2u       /* multiply the PoS weight by the advertised spare-capacity fraction */
+#define WWWS_FLAG_PUSH_PULL 8u  /* gossip as a full pairwise exchange: the pulled partner also merges the puller's
+                                   view (Appendix "Gossip-Driven Peer Synchronization": two nodes exchange views) */
 #define WWWS_FLAG_GREEDY 4u     /* customised rule: instead of drawing in proportion to the weights, take the
                                    candidate with the highest weight (lowest id on ties), then the next one on
                                    refusal; flags bit 0 then marks a runner-up within 1e-5 (relative) of the pick */

@@ -353,6 +353,12 @@ void orc_gossip_round(orc_net *n)
                     for (uint32_t col = 0; col < N; ++col) row[col] = orc_merge(row[col], prow[col]);
                     /* the pull itself tells the partner about the puller */
                     Vn[(size_t)p * N + i] = orc_merge(Vn[(size_t)p * N + i], self[i]);
+                    /* full pairwise exchange (flag 8): the partner also reconciles with the puller's view */
+                    if (c->flags & 8) {
+                        const uint64_t *irow = &V[(size_t)i * N];
+                        uint64_t *pnew = &Vn[(size_t)p * N];
+                        for (uint32_t col = 0; col < N; ++col) pnew[col] = orc_merge(pnew[col], irow[col]);
+                    }
                 }
             }
         }

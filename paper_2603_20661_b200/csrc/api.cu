@@ -105,6 +105,8 @@ void carve(const wwws_config& c, Carver& cv, Net& d, Staging& sg)
     d.d_backlog = cv.take<long long>(NP);
     d.w_led = cv.take<float>(NP);
     d.self_entry = cv.take<uint64_t>(NP); d.partner = cv.take<int32_t>(NP * 4);
+    d.in_deg = cv.take<uint32_t>(NP); d.in_off = cv.take<uint32_t>(NP); d.in_cursor = cv.take<uint32_t>(NP);
+    d.pullers = cv.take<int32_t>(NP * 4);
     d.cont = cv.take<uint2>(Rp * uint64_t(c.max_batch));
     d.rank_cdf = c.n_rank ? cv.take<uint32_t>(c.n_rank) : nullptr;
     d.stats = cv.take<unsigned long long>(Rp * sCount);
@@ -437,7 +439,7 @@ uint32_t wwws_profile_kernels(void) { return kKernelCount; }
 const char* wwws_profile_kernel_name(uint32_t k)
 {
     static const char* names[kKernelCount] = { "k_peer_init", "k_view_init", "k_advance", "k_fold", "k_finalize_check",
-        "k_rederive", "k_credit_total", "k_gossip_peer", "k_gossip_merge", "k_gossip_fixup", "k_dispatch", "k_duel",
+        "k_rederive", "k_credit_total", "k_gossip_peer", "k_gossip_merge", "k_gossip_fixup", "k_gossip_lists", "k_dispatch", "k_duel",
         "k_settle", "k_step_fused" };
     return k < kKernelCount ? names[k] : "";
 }

@@ -41,6 +41,7 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
         }
     }
     n.self_entry[x] = self;
+    n.in_deg[x] = 0;
     *reinterpret_cast<int4*>(n.partner + x * 4) = make_int4(part[0], part[1], part[2], part[3]);
 }
 
@@ -82,10 +83,14 @@ __device__ __forceinline__ void join(Q4& x, const Q4& y)
 // panel and walks kMergeIters rows of the block's row group.  Prologue: every row of the group
 // resolves its sources once (partner rows that answered, -1 otherwise) into shared memory, so
 // the streaming part has no dependent metadata loads.
-__global__ void __launch_bounds__(kMergeThreads, 8) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
+// PUSH: full pairwise exchange, a row also takes the old rows of the nodes that pulled it
+// (their ids come from the per-round reverse lists).
+template <bool PUSH>
+__global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
                                                                      uint32_t n_panels, uint32_t groups_per_panel)
 {
     __shared__ int4 s_src[kMergeThreads / 8 * kMergeIters];
+    __shared__ uint2 s_in[PUSH ? kMergeThreads / 8 * kMergeIters : 1];   // (offset, count) of the row's pullers
     const uint32_t b = blockIdx.x;
     const uint32_t per_replica = n_panels * groups_per_panel;
     const uint32_t r = b / per_replica;
@@ -107,6 +112,8 @@ __global__ void __launch_bounds__(kMergeThreads, 8) k_gossip_merge(Net n, uint32
             src.w = p4.w >= 0 && on[p4.w] ? p4.w : -1;
         }
         s_src[threadIdx.x] = src;
+        if (PUSH) s_in[threadIdx.x] = row < n.N && n.online[rbase + row] ? make_uint2(n.in_off[rbase + row], n.in_deg[rbase + row])
+                                                                          : make_uint2(0, 0);
     }
     __syncthreads();
     const uint32_t c = panel * panel_cols + 4u * (threadIdx.x & ((1u << chunk_shift) - 1u));
@@ -130,7 +137,75 @@ __global__ void __launch_bounds__(kMergeThreads, 8) k_gossip_merge(Net n, uint32
         if (src.y >= 0) join(acc, v1);
         if (src.z >= 0) join(acc, v2);
         if (src.w >= 0) join(acc, v3);
+        if (PUSH) {
+            const uint2 in_list = s_in[lr];
+            const int32_t* who = n.pullers + rbase * 4 + in_list.x;
+            for (uint32_t j = 0; j < in_list.y; ++j) join(acc, ld32(in + uint64_t(uint32_t(who[j])) * ld8));
+        }
         st32_stream(out + uint64_t(row) * ld8, acc);
+    }
+}
+
+// Reverse lists for the pairwise exchange: who pulled each node this round.
+__global__ void k_gossip_indeg(Net n)
+{
+    const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n.N) return;
+    const size_t x = size_t(r) * n.N + i;
+    if (!n.online[x]) return;
+    const int4 p4 = *reinterpret_cast<const int4*>(n.partner + x * 4);
+    const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+        if (p[s] >= 0 && n.online[size_t(r) * n.N + p[s]]) atomicAdd(&n.in_deg[size_t(r) * n.N + p[s]], 1u);
+}
+
+// Exclusive prefix sum of the in-degrees of one replica (one block per replica).
+__global__ void __launch_bounds__(1024) k_gossip_scan(Net n)
+{
+    __shared__ uint32_t warp_sum[32];
+    __shared__ uint32_t carry;
+    const uint32_t r = blockIdx.x, lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (uint32_t base = 0; base < n.N; base += 1024) {
+        const uint32_t i = base + threadIdx.x;
+        const uint32_t v = i < n.N ? n.in_deg[size_t(r) * n.N + i] : 0;
+        uint32_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= uint32_t(o)) incl += t; }
+        if (lane == 31) warp_sum[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            uint32_t w = warp_sum[lane], wi = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, wi, o); if (lane >= uint32_t(o)) wi += t; }
+            warp_sum[lane] = wi - w;                                       // exclusive over warps
+        }
+        __syncthreads();
+        const uint32_t excl = carry + warp_sum[wid] + incl - v;
+        if (i < n.N) { n.in_off[size_t(r) * n.N + i] = excl; n.in_cursor[size_t(r) * n.N + i] = 0; }
+        __syncthreads();
+        if (threadIdx.x == 1023) carry = excl + v;
+        __syncthreads();
+    }
+}
+
+__global__ void k_gossip_fill(Net n)
+{
+    const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n.N) return;
+    const size_t x = size_t(r) * n.N + i;
+    if (!n.online[x]) return;
+    const int4 p4 = *reinterpret_cast<const int4*>(n.partner + x * 4);
+    const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        if (p[s] < 0) continue;
+        const size_t px = size_t(r) * n.N + p[s];
+        if (!n.online[px]) continue;
+        const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
+        n.pullers[size_t(r) * n.N * 4 + n.in_off[px] + k] = int32_t(i);
     }
 }
 
@@ -185,8 +260,16 @@ void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c)
     const uint32_t n_panels = (n.ld + pc - 1) / pc;
     const uint32_t groups = (n.N + rows_per_block - 1) / rows_per_block;
     const uint64_t blocks = uint64_t(n.Rp) * n_panels * groups;
-    { Timed t(c, kGossipMerge);
-      k_gossip_merge<<<uint32_t(blocks), kMergeThreads, 0, c.stream>>>(n, pc, shift, n_panels, groups); }
+    if (n.flags & 8u) {
+        { Timed t(c, kGossipLists); k_gossip_indeg<<<pg, 128, 0, c.stream>>>(n); }
+        { Timed t(c, kGossipLists); k_gossip_scan<<<n.Rp, 1024, 0, c.stream>>>(n); }
+        { Timed t(c, kGossipLists); k_gossip_fill<<<pg, 128, 0, c.stream>>>(n); }
+        Timed t(c, kGossipMerge);
+        k_gossip_merge<true><<<uint32_t(blocks), kMergeThreads, 0, c.stream>>>(n, pc, shift, n_panels, groups);
+    } else {
+        Timed t(c, kGossipMerge);
+        k_gossip_merge<false><<<uint32_t(blocks), kMergeThreads, 0, c.stream>>>(n, pc, shift, n_panels, groups);
+    }
     { Timed t(c, kGossipFixup); k_gossip_fixup<<<pg, 128, 0, c.stream>>>(n); }
 }
 

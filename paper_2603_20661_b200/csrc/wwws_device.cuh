@@ -50,6 +50,8 @@ struct Net {
     float* w_led;
     // gossip scratch: this round's self entries and chosen partners
     uint64_t* self_entry; int32_t* partner;     // partner is [Rp][N][4]
+    // reverse lists of the pairwise exchange: in-degree, list offset, fill cursor, puller ids [Rp][4N]
+    uint32_t* in_deg; uint32_t* in_off; uint32_t* in_cursor; int32_t* pullers;
     // dispatch -> duel continuation, [Rp][max_batch]
     uint2* cont; uint32_t max_batch;
     const uint32_t* rank_cdf;

@@ -8,7 +8,7 @@ namespace wwws {
 
 // Kernel classes, for launch counts and optional event timing.
 enum KernelId : int { kPeerInit, kViewInit, kAdvance, kFold, kFinalizeCheck, kRederive, kCreditTotal, kGossipPeer,
-                      kGossipMerge, kGossipFixup, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
+                      kGossipMerge, kGossipFixup, kGossipLists, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
 
 // When enabled, every launch is bracketed by two events on the launching stream; read()
 // synchronises and returns the summed device time per kernel class.

@@ -135,6 +135,26 @@ def test_determinism_and_replica_sharding():
     assert np.array_equal(g.stats()[:2], outs[0][3][2:4])
 
 
+@pytest.mark.parametrize("n_peers,k,churn", [(1100, 4, 60_000), (300, 2, 0), (40, 1, 200_000)])
+def test_push_pull_gossip_matches_oracle(n_peers, k, churn):
+    """Full pairwise exchange (flag 8): reverse lists + merge over a variable number of rows."""
+    wl = synth.make_workload("churn4k", n_replicas=2, n_requests=4000, n_peers=n_peers)
+    wl.settings.flags |= 8
+    wl.settings.fanout_k = k
+    wl.settings.p_leave_ppm = wl.settings.p_join_ppm = churn
+    g, o = _pair(wl)
+    for s in range(wl.n_steps):
+        first = s * wl.batch
+        g.advance_time(wl.step_now_ms(s)); o.advance_time(wl.step_now_ms(s))
+        for _ in range(2):                       # two rounds per step
+            g.gossip_round(); o.gossip_round()
+        assert_same_state(g, o, f"push-pull step {s} gossip")
+        g.dispatch_batch(first, wl.batch); o.dispatch_batch(first, wl.batch)
+        g.duel_judge(); o.duel_judge()
+        g.settle_credits(True); o.settle_credits(True)
+    assert_same_state(g, o, "push-pull end", upto=wl.n_requests)
+
+
 def test_edge_cases_match_oracle():
     """Degenerate networks: two peers, a single request, everybody offline, nobody willing,
     requester-only origin, ragged window, duel probability one with tiny candidate sets."""

@@ -187,3 +187,34 @@ def test_gossip_version_overflow_is_reported():
     assert o.error() == 0
     o.gossip_round()
     assert o.error() == 4
+
+
+def test_push_pull_exchange_is_symmetric_and_faster():
+    """Flag 8: both ends of an exchange reconcile (the appendix figure shows two nodes swapping
+    views).  After a round each end dominates the other's old row; versions stay honest and
+    monotone; updates spread in fewer rounds than with pulls alone."""
+    N, k = 96, 1
+    rounds = {}
+    for flags in (0, 8):
+        st, pa, _ = make_net(N, fanout_k=k, seed=4, flags=flags, init_stale_max=7)
+        o = Oracle(st, pa)
+        t_conv = None
+        for t in range(40):
+            old = o.view()[0]
+            o.gossip_round()
+            new = o.view()[0]
+            ver_true = o.table("ver")[0].astype(np.uint64)
+            assert np.all(new >= old) and np.all(entry_ver(new) <= ver_true[None, :])
+            if flags == 8:
+                # somebody's old row is dominated by row i: its partner's; and row i's old content
+                # reached that partner: new[p] >= old[i] for at least one p != i
+                off = ~np.eye(N, dtype=bool)
+                for i in range(0, N, 11):
+                    dom_pull = [p for p in range(N) if p != i and np.all((new[i] >= old[p])[off[i]])]
+                    dom_push = [p for p in dom_pull if np.all((new[p] >= old[i])[off[p]])]
+                    assert dom_pull and dom_push, i
+            stale = (ver_true[None, :].astype(np.int64) - entry_ver(new).astype(np.int64)).max()
+            if t_conv is None and t >= 8 and stale <= 2 * math.log2(N):
+                t_conv = t
+        rounds[flags] = (t_conv, stale)
+    assert rounds[8][1] < rounds[0][1], rounds       # steady-state staleness is lower with push-pull
