@@ -126,6 +126,7 @@ def run_gpu(args):
     wl = synth.make_workload(args.workload, seed=args.seed, replica_offset=off, n_replicas=args.replicas)
     if args.batch:
         wl.batch = args.batch
+    wl.settings.flags |= (8 if args.push_pull else 0) | (4 if args.greedy else 0)
     st = wl.settings
     net = Network(st, wl.peers, wl.batch, device=dev)
     net.bind_requests(wl.requests, scores=False)
@@ -227,7 +228,7 @@ def run_gpu(args):
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u64 views, i64 ledgers, fp32 scores", "data": "synthetic",
             "config": {"workload": args.workload, "n_peers": st.n_peers, "n_replicas_per_gpu": Rp,
-                       "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "gossip_every": wl.gossip_every,
+                       "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "flags": st.flags, "gossip_every": wl.gossip_every,
                        "fanout_k": st.fanout_k, "entry": "wwws_step (fused dispatch+duel+settle)",
                        "l2": "inputs larger than L2 (view buffers %.1f GB per GPU)" % (2 * 8 * st.n_peers ** 2 * Rp / 1e9)},
             "clocks": clocks,
@@ -298,6 +299,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--replicas", type=int, default=None, help="override the workload's replica count (profiling)")
+    ap.add_argument("--push-pull", action="store_true", help="gossip as a full pairwise exchange (flag 8)")
+    ap.add_argument("--greedy", action="store_true", help="greedy dispatch rule instead of the proportional draw (flag 4)")
     ap.add_argument("--batch", type=int, default=None, help="override requests per replica per step (saturation runs)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
