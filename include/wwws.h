@@ -233,6 +233,18 @@ wwws_status wwws_import_table(wwws_network* net, wwws_table table, const void* h
 wwws_status wwws_export_view_rows(wwws_network* net, uint32_t replica, uint32_t row_first, uint32_t n_rows,
                                   uint64_t* host_dst);
 
+/* Checkpoint / resume.  A network's state is its per-peer tables (wwws_export_table), its view
+ * matrices (wwws_export_view_rows), its counters (wwws_stats; the chain head lives there) and its
+ * clock (simulated time and gossip round number).  Importing all of them into a network created
+ * from the same configuration and peer arrays continues the run bit for bit.  host_src of
+ * wwws_import_view_rows is n_rows * n_peers packed entries; host_src of wwws_import_stats is
+ * HOST [n_replicas] (the totals record is not read).  None of these may be called inside a batch. */
+wwws_status wwws_import_view_rows(wwws_network* net, uint32_t replica, uint32_t row_first, uint32_t n_rows,
+                                  const uint64_t* host_src);
+wwws_status wwws_export_clock(wwws_network* net, uint32_t* now_ms, uint32_t* round);
+wwws_status wwws_import_clock(wwws_network* net, uint32_t now_ms, uint32_t round);
+wwws_status wwws_import_stats(wwws_network* net, const wwws_stats_t* host_src);
+
 /* Kernels launched so far on behalf of this network. */
 uint64_t wwws_kernel_launches(const wwws_network* net);
 

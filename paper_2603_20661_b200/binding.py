@@ -29,7 +29,8 @@ EXPORTS = ("wwws_workspace_bytes", "wwws_create_network", "wwws_destroy_network"
            "wwws_advance_time", "wwws_gossip_round", "wwws_dispatch_batch", "wwws_duel_judge", "wwws_settle_credits",
            "wwws_step", "wwws_step_host", "wwws_stats", "wwws_export_table", "wwws_import_table",
            "wwws_export_view_rows", "wwws_kernel_launches", "wwws_last_error", "wwws_profile", "wwws_profile_read",
-           "wwws_profile_kernels", "wwws_profile_kernel_name", "wwws_gossip_round_static")
+           "wwws_profile_kernels", "wwws_profile_kernel_name", "wwws_gossip_round_static", "wwws_import_view_rows",
+           "wwws_export_clock", "wwws_import_clock", "wwws_import_stats")
 
 
 class WwwsError(RuntimeError):
@@ -93,6 +94,8 @@ def load():
             "wwws_stats": [vp, vp], "wwws_export_table": [vp, i32, vp, u64], "wwws_import_table": [vp, i32, vp, u64],
             "wwws_export_view_rows": [vp, u32, u32, u32, vp],
             "wwws_profile": [vp, i32], "wwws_profile_read": [vp, vp, vp],
+            "wwws_import_view_rows": [vp, u32, u32, u32, vp], "wwws_export_clock": [vp, C.POINTER(u32), C.POINTER(u32)],
+            "wwws_import_clock": [vp, u32, u32], "wwws_import_stats": [vp, vp],
         }
         for name, args in sig.items():
             f = getattr(L, name); f.argtypes = args; f.restype = C.c_int
@@ -284,6 +287,24 @@ class Network:
 
     def view(self):
         return np.stack([self.view_rows(r) for r in range(self.Rp)])
+
+    def checkpoint(self):
+        """Everything needed to resume: tables, views, counters, clock (host copies)."""
+        now, rnd = C.c_uint32(), C.c_uint32()
+        self._check(load().wwws_export_clock(self._h, C.byref(now), C.byref(rnd)), self._h)
+        return {"tables": {k: self.table(k) for k in TABLES}, "view": self.view(), "stats": self.stats()[:-1].copy(),
+                "clock": (now.value, rnd.value)}
+
+    def restore(self, ck):
+        """Load a checkpoint taken from a network of the same configuration."""
+        for k, v in ck["tables"].items():
+            self.import_table(k, v)
+        for r in range(self.Rp):
+            rows = np.ascontiguousarray(ck["view"][r], np.uint64)
+            self._check(load().wwws_import_view_rows(self._h, r, 0, self.N, rows.ctypes.data), self._h)
+        st = np.ascontiguousarray(ck["stats"], np.uint64)
+        self._check(load().wwws_import_stats(self._h, st.ctypes.data), self._h)
+        self._check(load().wwws_import_clock(self._h, *ck["clock"]), self._h)
 
     def results(self):
         self._torch.cuda.synchronize(self.device)

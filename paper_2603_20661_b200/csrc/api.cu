@@ -415,6 +415,45 @@ wwws_status wwws_export_view_rows(wwws_network* n, uint32_t replica, uint32_t ro
     return check_device_error(n);
 }
 
+wwws_status wwws_import_view_rows(wwws_network* n, uint32_t replica, uint32_t row_first, uint32_t n_rows, const uint64_t* host_src)
+{
+    if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    if (!host_src) return fail(n, WWWS_ERR_ARG, "host_src is NULL");
+    if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
+    if (replica >= n->d.Rp || uint64_t(row_first) + n_rows > n->d.N) return fail(n, WWWS_ERR_ARG, "rows out of range");
+    if (n_rows == 0) return WWWS_OK;
+    uint64_t* dst = n->d.view + (uint64_t(replica) * n->d.N + row_first) * n->d.ld;
+    CUDA_TRY(n, cudaMemcpy2DAsync(dst, n->d.ld * 8ull, host_src, n->d.N * 8ull, n->d.N * 8ull, n_rows, cudaMemcpyHostToDevice, n->stream));
+    CUDA_TRY(n, cudaStreamSynchronize(n->stream));
+    return WWWS_OK;
+}
+
+wwws_status wwws_export_clock(wwws_network* n, uint32_t* now_ms, uint32_t* round)
+{
+    if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    if (!now_ms || !round) return fail(n, WWWS_ERR_ARG, "output pointer is NULL");
+    *now_ms = n->t_last_ms; *round = n->round;
+    return WWWS_OK;
+}
+
+wwws_status wwws_import_clock(wwws_network* n, uint32_t now_ms, uint32_t round)
+{
+    if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
+    n->t_last_ms = now_ms; n->round = round;
+    return WWWS_OK;
+}
+
+wwws_status wwws_import_stats(wwws_network* n, const wwws_stats_t* host_src)
+{
+    if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    if (!host_src) return fail(n, WWWS_ERR_ARG, "host_src is NULL");
+    if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
+    CUDA_TRY(n, cudaMemcpyAsync(n->d.stats, host_src, uint64_t(n->d.Rp) * sizeof(wwws_stats_t), cudaMemcpyHostToDevice, n->stream));
+    CUDA_TRY(n, cudaStreamSynchronize(n->stream));
+    return WWWS_OK;
+}
+
 uint64_t wwws_kernel_launches(const wwws_network* n) { return n ? n->launches : 0; }
 
 wwws_status wwws_profile(wwws_network* n, int enable)
