@@ -31,6 +31,12 @@ UNIT = "requests/s"
 DEFAULT_WORKLOAD = "adversarial16k"          # the largest single-GPU configuration
 
 
+# DRAM traffic (read + write) of one k_gossip_merge pass over one replica, from the ncu capture
+# summarised in profiles/k_gossip_merge_adversarial16k_1replica.md; a launch over Rp replicas is
+# Rp such passes back to back (replica-major grid), so traffic scales with the replica count.
+NCU_MERGE_TRAFFIC = {"n_peers": 16384, "fanout_k": 4, "flags": 3, "bytes_per_replica": 2.1932e9 + 2.1138e9}
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -190,6 +196,8 @@ def run_gpu(args):
                 "ms_per_launch": t * 1e3}
 
     roof_merge = roof("k_gossip_merge", g_bytes)
+    if roof_merge and (st.n_peers, st.fanout_k, st.flags) == tuple(NCU_MERGE_TRAFFIC[k] for k in ("n_peers", "fanout_k", "flags")):
+        roof_merge["traffic"] = NCU_MERGE_TRAFFIC["bytes_per_replica"] * Rp
     if roof_merge:      # context: bytes a merge without L2 reuse would move (k+1 rows read, one written)
         roof_merge["bytes_per_launch_without_reuse"] = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
     roof_req = roof("k_step_fused", req_bytes / max(1, prof.get("k_step_fused", (0, 1))[1]))
