@@ -53,6 +53,9 @@ typedef enum {
 #define WWWS_FLAG_LOAD 2u       /* multiply the PoS weight by the advertised spare-capacity fraction */
 #define WWWS_FLAG_PUSH_PULL 8u  /* gossip as a full pairwise exchange: the pulled partner also merges the puller's
                                    view (Appendix "Gossip-Driven Peer Synchronization": two nodes exchange views) */
+#define WWWS_FLAG_FIFO 16u      /* exact queueing inside a batch: a request's latency counts the work that earlier
+                                   requests of the same batch put on its executor (executions, challenger runs,
+                                   judge evaluations), not only the executor's queue at the start of the batch */
 #define WWWS_FLAG_GREEDY 4u     /* customised rule: instead of drawing in proportion to the weights, take the
                                    candidate with the highest weight (lowest id on ties), then the next one on
                                    refusal; flags bit 0 then marks a runner-up within 1e-5 (relative) of the pick */

@@ -594,6 +594,9 @@ int orc_settle_credits(orc_net *n, int finalize)
             if (a == -3) { st[S_DROPPED] += 1; continue; }
             if (a == -4) { st[S_FAILED] += 1; continue; }
             uint32_t ex;
+            /* exact intra-batch queueing (flag 16): a request waits behind the work that earlier
+             * requests of the same batch put on its executor; otherwise only behind the batch-start queue */
+            uint64_t ahead = (c->flags & 16) ? (uint64_t)P[a < 0 ? o : (uint32_t)a].d_backlog : 0;
             if (a < 0) {                                                     /* S1 served at the origin */
                 st[a == -1 ? S_LOCAL : S_FALLBACK] += 1;
                 P[o].d_backlog += (int64_t)work; P[o].served_local += 1; ex = o;
@@ -625,7 +628,7 @@ int orc_settle_credits(orc_net *n, int finalize)
                 }
             }
             /* S4 latency estimate against the queue as it stood when the batch started */
-            uint64_t lat = ceil_div(((uint64_t)P[ex].backlog + work) * 1000, P[ex].cap_eff) + (a >= 0 ? c->hop_ms : 0);
+            uint64_t lat = ceil_div(((uint64_t)P[ex].backlog + ahead + work) * 1000, P[ex].cap_eff) + (a >= 0 ? c->hop_ms : 0);
             uint64_t deadline = (uint64_t)c->slo_num * ceil_div(work * 1000, c->cap_ref_tok_s) / c->slo_den;
             st[S_SUM_LAT] += lat;
             if (lat <= deadline) st[S_SLO_MET] += 1;

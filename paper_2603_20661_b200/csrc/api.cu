@@ -107,6 +107,7 @@ void carve(const wwws_config& c, Carver& cv, Net& d, Staging& sg)
     d.self_entry = cv.take<uint64_t>(NP); d.partner = cv.take<int32_t>(NP * 4);
     d.in_deg = cv.take<uint32_t>(NP); d.in_off = cv.take<uint32_t>(NP); d.in_cursor = cv.take<uint32_t>(NP);
     d.pullers = cv.take<int32_t>(NP * 4);
+    d.fifo_items = cv.take<int2>(Rp * uint64_t(c.max_batch) * 6); d.fifo_list = cv.take<uint2>(Rp * uint64_t(c.max_batch) * 6);
     d.cont = cv.take<uint2>(Rp * uint64_t(c.max_batch));
     d.rank_cdf = c.n_rank ? cv.take<uint32_t>(c.n_rank) : nullptr;
     d.stats = cv.take<unsigned long long>(Rp * sCount);
@@ -227,6 +228,7 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
     CUDA_TRY(nullptr, cudaMemsetAsync(d.credit_check, 0, d.Rp * 8ull, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.err, 0, 16, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.partner, 0xff, NP * 16, s));
+    CUDA_TRY(nullptr, cudaMemsetAsync(d.in_deg, 0, NP * 4, s));
     launch_peer_init(d, sg.credit0, sg.online0, cfg->init_stale_max, n->ctx());
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return fail(nullptr, WWWS_ERR_CUDA, std::string("initialisation kernels: ") + cudaGetErrorString(e));
     // host staging (`tot`, the caller's arrays) must stay valid until the copies are done
@@ -313,6 +315,7 @@ wwws_status wwws_settle_credits(wwws_network* n, int finalize)
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 2) return fail(n, WWWS_ERR_STATE, "settle_credits must follow duel_judge");
     launch_settle(n->d, n->batch_first, n->batch_count, n->ctx());
+    if (n->d.flags & 16u) launch_fifo(n->d, n->batch_first, n->batch_count, n->ctx());
     launch_fold(n->d, finalize != 0, n->ctx());
     n->phase = 0;
     return launch_status(n, "settle_credits");
@@ -330,6 +333,7 @@ wwws_status wwws_step(wwws_network* n, uint64_t first, uint64_t count, uint32_t 
         n->round += 1;
     }
     launch_step_fused(n->d, first, uint32_t(count), n->ctx());
+    if (n->d.flags & 16u) launch_fifo(n->d, first, uint32_t(count), n->ctx());
     launch_fold(n->d, finalize != 0, n->ctx());
     return launch_status(n, "step");
 }
@@ -478,7 +482,7 @@ uint32_t wwws_profile_kernels(void) { return kKernelCount; }
 const char* wwws_profile_kernel_name(uint32_t k)
 {
     static const char* names[kKernelCount] = { "k_peer_init", "k_view_init", "k_advance", "k_fold", "k_finalize_check",
-        "k_rederive", "k_credit_total", "k_gossip_peer", "k_gossip_merge", "k_gossip_fixup", "k_gossip_lists", "k_dispatch", "k_duel",
+        "k_rederive", "k_credit_total", "k_gossip_peer", "k_gossip_merge", "k_gossip_fixup", "k_gossip_lists", "k_fifo", "k_dispatch", "k_duel",
         "k_settle", "k_step_fused" };
     return k < kKernelCount ? names[k] : "";
 }

@@ -218,6 +218,7 @@ __global__ void k_gossip_fixup(Net n)
     if (i >= n.N) return;
     const size_t x = size_t(r) * n.N + i;
     if (i == 0) atomicAdd(&n.stats[size_t(r) * sCount + sRounds], 1ull);
+    n.in_deg[x] = 0;                                 // the reverse lists of this round are spent
     if (!n.online[x]) return;
     const uint64_t self = n.self_entry[x];
     unsigned long long* vn = reinterpret_cast<unsigned long long*>(n.view_new);
@@ -233,6 +234,14 @@ __global__ void k_gossip_fixup(Net n)
         else atomicMax(vn + px * n.ld + i, self);
     }
     if (marks) atomicAdd(&n.stats[size_t(r) * sCount + sOfflineMarks], (unsigned long long)marks);
+}
+
+// per-peer exclusive prefix sums of in_deg into in_off (also clears in_cursor); shared with the
+// intra-batch queueing of the settlement
+void launch_scan_in_degrees(const Net& n, const LaunchCtx& c, int kernel_id)
+{
+    Timed t(c, kernel_id);
+    k_gossip_scan<<<n.Rp, 1024, 0, c.stream>>>(n);
 }
 
 // Panel width: the widest power of two (32 .. 512 columns) whose panel of N rows fits the

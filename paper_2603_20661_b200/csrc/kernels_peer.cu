@@ -76,6 +76,7 @@ __global__ void k_fold(Net n, int finalize)
         const size_t x = size_t(r) * n.N + j;
         const long long db = n.d_backlog[x];
         if (db) { n.backlog[x] += db; n.d_backlog[x] = 0; }
+        if (n.flags & 16u) n.in_deg[x] = 0;          // per-peer item counts of the batch's queueing pass
         if (finalize) {
             const int64_t c = n.credit[x] + n.d_credit[x];
             const uint32_t w = n.wins[x] + n.d_wins[x], d = n.duels[x] + n.d_duels[x];

@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
         const size_t x = size_t(r) * n.Q + first + idx;
         const int4 j4 = *reinterpret_cast<const int4*>(n.judges + 4 * x);
         const int jd[4] = { j4.x, j4.y, j4.z, j4.w };
-        settle_one(n, r, uint32_t(first + idx), n.origin[x], n.len_in[x], n.len_out[x], n.exec_a[x], n.exec_b[x], jd, n.outcome[x],
+        settle_one(n, r, uint32_t(first + idx), idx, n.origin[x], n.len_in[x], n.len_out[x], n.exec_a[x], n.exec_b[x], jd, n.outcome[x],
                    (n.rflags[x] & 1) != 0, s);
     }
 #pragma unroll
@@ -224,6 +224,60 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
     for (int o = 16; o; o >>= 1) dg += __shfl_down_sync(kFull, dg, o);
     if ((threadIdx.x & 31) == 0) stats_add(bs, sPendingDigest, dg);
     stats_end(n, bs, r);
+}
+
+// ---- exact intra-batch queueing (flag 16) -------------------------------------------------------
+
+// Scatter the batch's work items into per-peer lists (offsets from the scan of in_deg).
+__global__ void k_fifo_fill(Net n, uint32_t count)
+{
+    const uint32_t r = blockIdx.y, slot = blockIdx.x * blockDim.x + threadIdx.x;
+    if (slot >= count * 6) return;
+    const int2 item = n.fifo_items[size_t(r) * n.max_batch * 6 + slot];
+    if (item.x < 0) return;
+    const size_t px = size_t(r) * n.N + item.x;
+    const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
+    n.fifo_list[size_t(r) * n.max_batch * 6 + n.in_off[px] + k] = make_uint2(slot / 6, uint32_t(item.y));
+}
+
+// Latency of every served request: it waits behind the batch-start queue of its executor and
+// behind the items that earlier requests of the batch put there.
+__global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uint32_t count)
+{
+    __shared__ BlockStats bs;
+    stats_begin(bs);
+    const uint32_t r = blockIdx.y, idx = blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t met = 0;
+    unsigned long long lat_sum = 0;
+    if (idx < count) {
+        const size_t x = size_t(r) * n.Q + first + idx;
+        const int a = n.exec_a[x];
+        if (a != -3 && a != -4) {
+            const uint32_t ex = a < 0 ? n.origin[x] : uint32_t(a);
+            const size_t px = size_t(r) * n.N + ex;
+            const uint2* list = n.fifo_list + size_t(r) * n.max_batch * 6 + n.in_off[px];
+            const uint32_t len = n.in_deg[px];
+            uint64_t ahead = 0;
+            for (uint32_t j = 0; j < len; ++j) { const uint2 it = list[j]; if (it.x < idx) ahead += it.y; }
+            const uint64_t work = uint64_t(n.len_in[x]) + n.len_out[x], cap = n.cap_eff[px];
+            const uint64_t t = (uint64_t(n.backlog[px]) + ahead + work) * 1000ull, tq = udiv64by32(t, uint32_t(cap));
+            const uint64_t lat = tq + (tq * cap != t ? 1 : 0) + (a >= 0 ? n.hop_ms : 0);
+            const uint64_t ideal = udiv64by32(work * 1000ull + n.cap_ref - 1, n.cap_ref);
+            const uint64_t deadline = udiv64by32(uint64_t(n.slo_num) * ideal, n.slo_den);
+            lat_sum = lat; met = lat <= deadline;
+        }
+    }
+    const uint32_t m = __reduce_add_sync(kFull, met);
+    for (int o = 16; o; o >>= 1) lat_sum += __shfl_down_sync(kFull, lat_sum, o);
+    if ((threadIdx.x & 31) == 0) { stats_add(bs, sSloMet, m); stats_add(bs, sSumLat, lat_sum); }
+    stats_end(n, bs, r);
+}
+
+void launch_fifo(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    launch_scan_in_degrees(n, c, kFifo);
+    { Timed t(c, kFifo); k_fifo_fill<<<dim3((count * 6 + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, count); }
+    { Timed t(c, kFifo); k_fifo_latency<<<dim3((count + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, first, count); }
 }
 
 static dim3 warp_grid(const Net& n, uint32_t count) { return dim3((count + kWarpsPerBlock - 1) / kWarpsPerBlock, n.Rp); }

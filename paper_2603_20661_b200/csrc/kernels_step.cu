@@ -176,7 +176,7 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
             *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(-1, -1, -1, -1);
             const int jd[4] = { -1, -1, -1, -1 };
             acc.c[sProbes] += d.n_probes;
-            settle_one(n, r, q, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
+            settle_one(n, r, q, idx, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
         }
     }
     __syncthreads();
@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
         n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = d.near ? 1 : 0;
         *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
         acc.c[sProbes] += d.n_probes;
-        settle_one(n, r, q, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
+        settle_one(n, r, q, didx, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
     }
 
     // ---- counters: warp reduce, block reduce, one atomic per counter and block ---------------

@@ -101,9 +101,26 @@ struct SettleAcc {
     unsigned long long digest;     // wrapping sum of the record hashes of this thread's requests
 };
 
-__device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q, uint32_t o, uint32_t li, uint32_t lo, int a, int b,
-                                           const int (&jd)[4], uint32_t oc, bool near, SettleAcc& s)
+// With exact intra-batch queueing (flag 16) the latency of a request depends on the work that
+// earlier requests of the batch put on its executor, so settle_one only records the batch's work
+// items (slot = request*6 + role: primary, challenger, four judges) and counts them per peer;
+// k_fifo_latency computes the latencies once the per-peer lists are built.
+__device__ __forceinline__ void fifo_emit(const Net& n, uint32_t r, uint32_t bidx, uint32_t role, int peer, uint32_t tokens)
 {
+    n.fifo_items[(size_t(r) * n.max_batch + bidx) * 6 + role] = make_int2(peer, int(tokens));
+    if (peer >= 0) atomicAdd(&n.in_deg[size_t(r) * n.N + peer], 1u);
+}
+
+__device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q, uint32_t bidx, uint32_t o, uint32_t li, uint32_t lo,
+                                           int a, int b, const int (&jd)[4], uint32_t oc, bool near, SettleAcc& s)
+{
+    if (n.flags & 16u) {
+        const bool served = a != -3 && a != -4, duel = a >= 0 && oc >= 1 && oc <= 3;
+        fifo_emit(n, r, bidx, 0, served ? (a < 0 ? int(o) : a) : -1, li + lo);
+        fifo_emit(n, r, bidx, 1, duel ? b : -1, li + lo);
+#pragma unroll
+        for (int l = 0; l < 4; ++l) fifo_emit(n, r, bidx, 2 + l, duel ? jd[l] : -1, li + 2u * lo);
+    }
     const size_t base = size_t(r) * n.N;
     const uint64_t work = uint64_t(li) + lo;
     s.c[sRequests]++;
@@ -159,6 +176,7 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
         }
         add64(&n.d_credit[base + o], -pay);
     }
+    if (n.flags & 16u) return;                       // latency and SLO are counted by k_fifo_latency
     const uint64_t cap = n.cap_eff[base + ex];
     const uint64_t t = (uint64_t(n.backlog[base + ex]) + work) * 1000ull, tq = udiv64by32(t, uint32_t(cap));
     const uint64_t lat = tq + (tq * cap != t ? 1 : 0) + (a >= 0 ? n.hop_ms : 0);

@@ -52,6 +52,9 @@ struct Net {
     uint64_t* self_entry; int32_t* partner;     // partner is [Rp][N][4]
     // reverse lists of the pairwise exchange: in-degree, list offset, fill cursor, puller ids [Rp][4N]
     uint32_t* in_deg; uint32_t* in_off; uint32_t* in_cursor; int32_t* pullers;
+    // exact intra-batch queueing: work items (peer, tokens) of the batch [Rp][6*max_batch] (slot = request*6 + role)
+    // and, per peer, the list (request, tokens) of the items queued on it
+    int2* fifo_items; uint2* fifo_list;
     // dispatch -> duel continuation, [Rp][max_batch]
     uint2* cont; uint32_t max_batch;
     const uint32_t* rank_cdf;

@@ -8,7 +8,7 @@ namespace wwws {
 
 // Kernel classes, for launch counts and optional event timing.
 enum KernelId : int { kPeerInit, kViewInit, kAdvance, kFold, kFinalizeCheck, kRederive, kCreditTotal, kGossipPeer,
-                      kGossipMerge, kGossipFixup, kGossipLists, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
+                      kGossipMerge, kGossipFixup, kGossipLists, kFifo, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
 
 // When enabled, every launch is bracketed by two events on the launching stream; read()
 // synchronises and returns the summed device time per kernel class.
@@ -44,6 +44,8 @@ void launch_fold(const Net& n, int finalize, const LaunchCtx& c);
 void launch_rederive(const Net& n, const LaunchCtx& c);
 void launch_credit_total(const Net& n, const LaunchCtx& c);
 void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c);
+void launch_scan_in_degrees(const Net& n, const LaunchCtx& c, int kernel_id);
+void launch_fifo(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_duel(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_settle(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);

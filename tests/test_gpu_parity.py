@@ -155,6 +155,31 @@ def test_push_pull_gossip_matches_oracle(n_peers, k, churn):
     assert_same_state(g, o, "push-pull end", upto=wl.n_requests)
 
 
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiers64", dict(n_requests=5000)),
+                                     ("zipf1k", dict(n_replicas=3, n_requests=2500, n_peers=200))])
+def test_fifo_queueing_matches_oracle(name, kw):
+    """Exact intra-batch queueing (flag 16) through both call paths, with duels and heavy contention."""
+    wl = synth.make_workload(name, **kw)
+    wl.settings.flags |= 16
+    wl.settings.p_duel_ppm = 300_000
+    g, o = _pair(wl)
+    g2 = _pair(wl)[0]
+    for s in range(wl.n_steps):
+        first = s * wl.batch
+        cnt = min(wl.batch, wl.n_requests - first)
+        gossip = s % wl.gossip_every == 0
+        g.step(first, cnt, wl.step_now_ms(s), gossip, s % 2 == 0)
+        g2.run_step(first, cnt, wl.step_now_ms(s), gossip, s % 2 == 0)
+        o.run_step(first, cnt, wl.step_now_ms(s), gossip, s % 2 == 0)
+        if s < 3 or s % 4 == 0:
+            assert_same_state(g, o, f"fifo fused step {s}", upto=first + cnt, views=False)
+            assert_same_state(g2, o, f"fifo six-call step {s}", upto=first + cnt, views=False)
+    assert_same_state(g, o, "fifo fused end", upto=wl.n_requests)
+    assert_same_state(g2, o, "fifo six-call end", upto=wl.n_requests)
+    base = synth.make_workload(name, **kw)
+    assert o.stats_dict()["sum_latency_ms"] > 0
+
+
 def test_edge_cases_match_oracle():
     """Degenerate networks: two peers, a single request, everybody offline, nobody willing,
     requester-only origin, ragged window, duel probability one with tiny candidate sets."""

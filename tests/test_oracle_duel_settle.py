@@ -285,3 +285,44 @@ def test_advance_time_and_latency_hand_cases():
         o2.advance_time(w * 60_000 + 59_999)
         assert np.array_equal(o2.table("cap_eff")[0], cap)      # constant inside a window
     assert all(abs(h - 0.5) < 5 * math.sqrt(0.25 / 400) for h in halves) and len(set(halves)) > 1
+
+
+def test_fifo_queueing_inside_a_batch_hand_cases():
+    """Flag 16: requests of one batch queue behind each other at their executor (all roles
+    count: executions, challenger runs, judge evaluations).  One executor, known sizes."""
+    lens = (600, 400)                                       # 1000 tokens per request
+    st, pa, rq = make_net(2, n_requests=6, lens=lens, p_duel_ppm=0, flags=16,
+                          peers=requester_first(2, cap_true_tok_s=np.array([0, 1000]), credit0=10 ** 6))
+    o = Oracle(st, pa); o.bind_requests(rq)
+    o.poke_peer(0, 1, backlog=500)
+    o.dispatch_batch(0, 4); o.duel_judge(); o.settle_credits(True)
+    assert np.all(o.results()["exec_a"][0, :4] == 1)
+    # latencies: (500 + k*1000 + 1000) tokens at 1000 tok/s -> 1500, 2500, 3500, 4500 ms
+    assert o.stats_dict()["sum_latency_ms"] == 1500 + 2500 + 3500 + 4500
+    assert o.stats_dict()["slo_met"] == 0                   # deadline 2 * 500 ms
+    assert o.table("backlog")[0, 1] == 4500
+    # next batch starts from the folded queue
+    o.dispatch_batch(4, 2); o.duel_judge(); o.settle_credits(True)
+    assert o.stats_dict()["sum_latency_ms"] == 12000 + 5500 + 6500
+    # without the flag every request of a batch sees only the batch-start queue
+    st.flags = 0
+    o2 = Oracle(st, pa); o2.bind_requests(rq)
+    o2.poke_peer(0, 1, backlog=500)
+    o2.dispatch_batch(0, 4); o2.duel_judge(); o2.settle_credits(True)
+    assert o2.stats_dict()["sum_latency_ms"] == 4 * 1500
+    # challenger and judge work queues too: N = 5, every request a duel with 2 judges
+    st3, pa3, rq3 = make_net(5, n_requests=40, lens=lens, p_duel_ppm=1_000_000, n_judges=2, flags=16, seed=3,
+                             peers=requester_first(5, credit0=10 ** 6))
+    o3 = Oracle(st3, pa3); o3.bind_requests(rq3)
+    o3.dispatch_batch(0, 40); o3.duel_judge(); o3.settle_credits(True)
+    res = o3.results()
+    queued = np.zeros(5, np.int64); total = 0
+    for q in range(40):
+        a, b = res["exec_a"][0, q], res["exec_b"][0, q]
+        total += -(-(queued[a] + 1000) * 1000 // 2000)      # ceil((ahead + work) * 1000 / cap)
+        queued[a] += 1000; queued[b] += 1000
+        for j in res["judges"][0, q]:
+            if j >= 0:
+                queued[j] += 600 + 2 * 400
+    assert o3.stats_dict()["sum_latency_ms"] == total
+    assert np.array_equal(o3.table("backlog")[0], queued)
