@@ -202,6 +202,10 @@ def run_gpu(args):
         roof_merge["bytes_per_launch_without_reuse"] = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
     roof_req = roof("k_step_fused", req_bytes / max(1, prof.get("k_step_fused", (0, 1))[1]))
     roofline = roof_merge if dom == "k_gossip_merge" else roof_req
+    # requests/s of dispatch+duel+settle alone (advance, fused step, fold, block commit), from the same events
+    t_req = sum(prof[k][0] for k in ("k_advance", "k_step_fused", "k_fold", "k_finalize_check", "k_fifo") if k in prof)
+    req_only = {"value": delta_b["n_requests"] / (t_req * 1e-3), "unit": UNIT, "ms_per_step": t_req / K,
+                "kernels": "k_advance + k_step_fused + k_fold + k_finalize_check, summed CUDA-event time"}
 
     # ---- region C: end to end through host buffers ---------------------------------------------
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
@@ -245,6 +249,7 @@ def run_gpu(args):
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_request_path": roof_req,
+            "dispatch_duel_settle_only": req_only,
             "roofline_gossip_merge": roof_merge,
             "kernels": kernels,
             "step_mix": {k: delta[k] for k in ("n_requests", "n_delegated", "n_duel", "n_probes", "rounds")},
@@ -255,12 +260,12 @@ def run_gpu(args):
     return line
 
 
-def oracle_run(workload, seed, steps, warmup, replicas=1):
+def oracle_run(workload, seed, steps, warmup, replicas=1, first_replica=0):
     """Time the CPU oracle, as it stands, on `replicas` replicas of the workload: `warmup`
     untimed steps, then `steps` timed ones.  Returns (requests/s, seconds, description)."""
     from oracle import Oracle
     from paper_2603_20661_b200 import synth
-    wl = synth.slice_replicas(synth.make_workload(workload, seed=seed), 0, replicas)
+    wl = synth.slice_replicas(synth.make_workload(workload, seed=seed), first_replica, first_replica + replicas)
     o = Oracle(wl.settings, wl.peers)
     o.bind_requests(wl.requests)
     s = 0
@@ -277,6 +282,32 @@ def oracle_run(workload, seed, steps, warmup, replicas=1):
             f"single thread")
     o.close()
     return n / dt, dt, desc
+
+
+def _oracle_worker(job):
+    workload, seed, steps, replica = job
+    v, dt, _ = oracle_run(workload, seed, steps, 0, 1, replica)
+    return v * dt, dt
+
+
+def oracle_all_cores(workload, seed, steps):
+    """One independent oracle instance per host core, each on its own replica (replicas share
+    nothing); processes are started with `spawn`.  Returns (requests/s, workers, seconds)."""
+    import multiprocessing as mp
+    from paper_2603_20661_b200 import synth
+    wl = synth.make_workload(workload, seed=seed, n_requests=1)
+    view_bytes = 2 * 8 * wl.settings.n_peers ** 2 + (64 << 20)
+    try:
+        import psutil
+        fit = max(1, int(psutil.virtual_memory().available * 0.6 // view_bytes))
+    except ImportError:
+        fit = 4
+    workers = max(1, min(os.cpu_count() or 1, wl.settings.n_replicas, fit))
+    t0 = time.perf_counter()
+    with mp.get_context("spawn").Pool(workers) as pool:
+        out = pool.map_async(_oracle_worker, [(workload, seed, steps, r) for r in range(workers)]).get(timeout=240)
+    wall = time.perf_counter() - t0
+    return sum(n for n, _ in out) / max(dt for _, dt in out), workers, wall
 
 
 def run_reference(args):
@@ -311,7 +342,8 @@ def main():
     ap.add_argument("--greedy", action="store_true", help="greedy dispatch rule instead of the proportional draw (flag 4)")
     ap.add_argument("--batch", type=int, default=None, help="override requests per replica per step (saturation runs)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
-    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing legs")
+    ap.add_argument("--no-cpu-all-cores", action="store_true", help="skip the one-oracle-per-core timing leg")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -326,6 +358,14 @@ def main():
             from paper_2603_20661_b200 import synth
             ge = synth.make_workload(args.workload, n_replicas=1, n_requests=1000).gossip_every
             v, dt, desc = oracle_run(args.workload, args.seed, ge, 0, 1)
+            if not args.no_cpu_all_cores:
+                try:
+                    va, workers, wall = oracle_all_cores(args.workload, args.seed, ge)
+                    line["cpu_baseline_all_cores"] = {
+                        "value": va, "unit": UNIT, "cores": workers, "kind": "oracle", "wall_seconds": wall,
+                        "sample": f"{workers} independent oracle instances, one replica each, same steps"}
+                except Exception as e:          # a baseline leg must never cost the GPU result
+                    line["cpu_baseline_all_cores"] = {"unavailable": repr(e)}
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
                                     "seconds": dt}
         print(json.dumps(line))

@@ -80,14 +80,18 @@ __device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, 
     return pick;
 }
 
-// D6: the drawn candidate answers by its true state and its own accept policy.
+// D6: the drawn candidate answers by its true state and its own accept policy.  All five values
+// are loaded at once and the probe's random word is computed while they are in flight: one
+// memory round trip per probe instead of a chain of dependent ones.
 __device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg, uint32_t q, uint32_t blk, int pick)
 {
     const size_t x = size_t(r) * n.N + kWin * blk + pick;
     const uint32_t cap = n.cap_eff[x];
-    if (!n.online[x] || cap == 0) return false;
-    if (util_at_least(cap, n.backlog[x], n.util_window_ms, n.accept_util_pm[x])) return false;
-    return ppm(draw(n, q, uint32_t(pick) >> 2, rg, kProbe).w[pick & 3]) < n.accept_ppm[x];
+    const uint8_t on = n.online[x];
+    const int64_t queued = n.backlog[x];
+    const uint32_t accept_util = n.accept_util_pm[x], accept_freq = n.accept_ppm[x];
+    const uint32_t u = ppm(draw(n, q, uint32_t(pick) >> 2, rg, kProbe).w[pick & 3]);
+    return on && cap != 0 && !util_at_least(cap, queued, n.util_window_ms, accept_util) && u < accept_freq;
 }
 
 template <int BT>

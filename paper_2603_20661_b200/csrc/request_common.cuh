@@ -77,11 +77,14 @@ __device__ __forceinline__ bool origin_offloads(const Net& n, uint32_t r, uint32
 {
     if (o >= n.N) { set_error(n, eArg, o); code = -3; return false; }
     const size_t ox = size_t(r) * n.N + o;
-    if (!n.online[ox]) { code = -3; return false; }
+    // independent loads first, decisions afterwards: one memory round trip
+    const uint8_t on = n.online[ox];
     const uint32_t cap = n.cap_eff[ox];
+    const int64_t queued = n.backlog[ox], credit = n.credit[ox];
+    const uint32_t thr = n.offload_util_pm[ox], freq = n.offload_ppm[ox];
+    if (!on) { code = -3; return false; }
     code = cap == 0 ? -4 : -1;
-    return util_at_least(cap, n.backlog[ox], n.util_window_ms, n.offload_util_pm[ox]) &&
-           ppm(rx.w[0]) < n.offload_ppm[ox] && n.credit[ox] >= n.R;
+    return util_at_least(cap, queued, n.util_window_ms, thr) && ppm(rx.w[0]) < freq && credit >= n.R;
 }
 
 // 64-bit by 32-bit unsigned division; the common case (numerator below 2^32) takes the short
