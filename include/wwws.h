@@ -55,7 +55,9 @@ typedef enum {
                                    view (Appendix "Gossip-Driven Peer Synchronization": two nodes exchange views) */
 #define WWWS_FLAG_FIFO 16u      /* exact queueing inside a batch: a request's latency counts the work that earlier
                                    requests of the same batch put on its executor (executions, challenger runs,
-                                   judge evaluations), not only the executor's queue at the start of the batch */
+                                   judge evaluations), not only the executor's queue at the start of the batch;
+                                   also validates every payment against the payer's balance inside the open block
+                                   (n_uncovered) */
 #define WWWS_FLAG_GREEDY 4u     /* customised rule: instead of drawing in proportion to the weights, take the
                                    candidate with the highest weight (lowest id on ties), then the next one on
                                    refusal; flags bit 0 then marks a runner-up within 1e-5 (relative) of the pick */
@@ -136,6 +138,8 @@ typedef struct {
                                 hash of the parent id, the block's operations digest and its height */
     uint64_t pending_digest; /* order-independent digest (wrapping sum of per-record hashes) of the credit
                                 operations settled since the last finalization */
+    uint64_t n_uncovered;    /* with WWWS_FLAG_FIFO: payments that exceeded the payer's finalized balance minus
+                                what it had already spent in the open block (double-spend check; counted only) */
 } wwws_stats_t;
 
 /* Per-peer tables for wwws_export_table / wwws_import_table; element type in the comment. */

@@ -109,11 +109,13 @@ typedef struct {
     int64_t d_credit; uint32_t d_wins, d_duels;
     /* backlog added by the batch being settled */
     int64_t d_backlog;
+    /* credits spent since the last finalization: in earlier batches of the block, in this batch so far */
+    int64_t blk_spent, d_spent;
 } peer_t;
 
 enum { S_REQUESTS, S_LOCAL, S_FALLBACK, S_DROPPED, S_FAILED, S_DELEGATED, S_DUEL, S_DUEL_CANCELLED, S_DRAW,
        S_JUDGE_EVALS, S_PROBES, S_NEAR, S_SLO_MET, S_SUM_LAT, S_OFFLINE_MARKS, S_ROUNDS, S_BLOCKS, S_CREDIT_TOTAL,
-       S_CHAIN_HEAD, S_PENDING_DIGEST, S_N };
+       S_CHAIN_HEAD, S_PENDING_DIGEST, S_UNCOVERED, S_N };
 
 typedef struct {
     uint32_t inplay;       /* lanes still in play after the draws so far */
@@ -602,6 +604,14 @@ int orc_settle_credits(orc_net *n, int finalize)
                 P[o].d_backlog += (int64_t)work; P[o].served_local += 1; ex = o;
             } else {                                                         /* S2 credits-for-offloading */
                 st[S_DELEGATED] += 1;
+                if (c->flags & 16) {
+                    /* in-block validation (Section "Credit-based Transaction System": a payer must not spend the
+                     * same credits twice): a payment is covered only by the payer's finalized balance minus what it
+                     * already spent in this block; earnings of the open block cannot be spent yet */
+                    int64_t pay = c->reward_R * ((n->outcome[x] >= 1 && n->outcome[x] <= 3) ? 2 : 1);
+                    if (P[o].credit - P[o].blk_spent - P[o].d_spent < pay) st[S_UNCOVERED] += 1;
+                    P[o].d_spent += pay;
+                }
                 post(n, r, (uint32_t)q, OP_PAY, o, -c->reward_R); post(n, r, (uint32_t)q, OP_EARN, (uint32_t)a, c->reward_R);
                 P[a].d_backlog += (int64_t)work; P[a].served += 1; ex = (uint32_t)a;
                 uint8_t oc = n->outcome[x];
@@ -633,7 +643,10 @@ int orc_settle_credits(orc_net *n, int finalize)
             st[S_SUM_LAT] += lat;
             if (lat <= deadline) st[S_SLO_MET] += 1;
         }
-        for (uint32_t j = 0; j < n->N; ++j) { P[j].backlog += P[j].d_backlog; P[j].d_backlog = 0; }
+        for (uint32_t j = 0; j < n->N; ++j) {
+            P[j].backlog += P[j].d_backlog; P[j].d_backlog = 0;
+            P[j].blk_spent = finalize ? 0 : P[j].blk_spent + P[j].d_spent; P[j].d_spent = 0;
+        }
         if (finalize) finalize_replica(n, r);
     }
     n->phase = 0;

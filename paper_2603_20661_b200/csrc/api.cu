@@ -107,7 +107,8 @@ void carve(const wwws_config& c, Carver& cv, Net& d, Staging& sg)
     d.self_entry = cv.take<uint64_t>(NP); d.partner = cv.take<int32_t>(NP * 4);
     d.in_deg = cv.take<uint32_t>(NP); d.in_off = cv.take<uint32_t>(NP); d.in_cursor = cv.take<uint32_t>(NP);
     d.pullers = cv.take<int32_t>(NP * 4);
-    d.fifo_items = cv.take<int2>(Rp * uint64_t(c.max_batch) * 6); d.fifo_list = cv.take<uint2>(Rp * uint64_t(c.max_batch) * 6);
+    d.fifo_items = cv.take<int2>(Rp * uint64_t(c.max_batch) * 7); d.fifo_list = cv.take<uint2>(Rp * uint64_t(c.max_batch) * 7);
+    d.blk_spent = cv.take<long long>(NP); d.d_spent = cv.take<long long>(NP);
     d.cont = cv.take<uint2>(Rp * uint64_t(c.max_batch));
     d.rank_cdf = c.n_rank ? cv.take<uint32_t>(c.n_rank) : nullptr;
     d.stats = cv.take<unsigned long long>(Rp * sCount);

@@ -30,6 +30,7 @@ __global__ void k_peer_init(Net n, const int64_t* __restrict__ credit0, const ui
     n.stake[x] = st;
     n.wins[x] = 0; n.duels[x] = 0; n.served[x] = 0; n.served_local[x] = 0;
     n.d_credit[x] = 0; n.d_wins[x] = 0; n.d_duels[x] = 0; n.d_backlog[x] = 0;
+    n.blk_spent[x] = 0; n.d_spent[x] = 0;
     n.w_led[x] = ledger_weight(n, st, 0, 0);
     n.self_entry[x] = 0;
 }
@@ -76,7 +77,11 @@ __global__ void k_fold(Net n, int finalize)
         const size_t x = size_t(r) * n.N + j;
         const long long db = n.d_backlog[x];
         if (db) { n.backlog[x] += db; n.d_backlog[x] = 0; }
-        if (n.flags & 16u) n.in_deg[x] = 0;          // per-peer item counts of the batch's queueing pass
+        if (n.flags & 16u) {
+            n.in_deg[x] = 0;                         // per-peer item counts of the batch's queueing pass
+            n.blk_spent[x] = finalize ? 0 : n.blk_spent[x] + n.d_spent[x];
+            n.d_spent[x] = 0;
+        }
         if (finalize) {
             const int64_t c = n.credit[x] + n.d_credit[x];
             const uint32_t w = n.wins[x] + n.d_wins[x], d = n.duels[x] + n.d_duels[x];

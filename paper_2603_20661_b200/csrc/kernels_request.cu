@@ -232,12 +232,13 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
 __global__ void k_fifo_fill(Net n, uint32_t count)
 {
     const uint32_t r = blockIdx.y, slot = blockIdx.x * blockDim.x + threadIdx.x;
-    if (slot >= count * 6) return;
-    const int2 item = n.fifo_items[size_t(r) * n.max_batch * 6 + slot];
+    if (slot >= count * 7) return;
+    const int2 item = n.fifo_items[size_t(r) * n.max_batch * 7 + slot];
     if (item.x < 0) return;
     const size_t px = size_t(r) * n.N + item.x;
     const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
-    n.fifo_list[size_t(r) * n.max_batch * 6 + n.in_off[px] + k] = make_uint2(slot / 6, uint32_t(item.y));
+    // entry: (request, amount), bit 31 of the amount marks a payment (role 6) as opposed to queued work
+    n.fifo_list[size_t(r) * n.max_batch * 7 + n.in_off[px] + k] = make_uint2(slot / 7, uint32_t(item.y) | (slot % 7 == 6 ? 0x80000000u : 0u));
 }
 
 // Latency of every served request: it waits behind the batch-start queue of its executor and
@@ -247,7 +248,7 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
     __shared__ BlockStats bs;
     stats_begin(bs);
     const uint32_t r = blockIdx.y, idx = blockIdx.x * blockDim.x + threadIdx.x;
-    uint32_t met = 0;
+    uint32_t met = 0, uncovered = 0;
     unsigned long long lat_sum = 0;
     if (idx < count) {
         const size_t x = size_t(r) * n.Q + first + idx;
@@ -255,10 +256,22 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
         if (a != -3 && a != -4) {
             const uint32_t ex = a < 0 ? n.origin[x] : uint32_t(a);
             const size_t px = size_t(r) * n.N + ex;
-            const uint2* list = n.fifo_list + size_t(r) * n.max_batch * 6 + n.in_off[px];
+            const uint2* list = n.fifo_list + size_t(r) * n.max_batch * 7 + n.in_off[px];
             const uint32_t len = n.in_deg[px];
             uint64_t ahead = 0;
-            for (uint32_t j = 0; j < len; ++j) { const uint2 it = list[j]; if (it.x < idx) ahead += it.y; }
+            for (uint32_t j = 0; j < len; ++j) { const uint2 it = list[j]; if (it.x < idx && !(it.y >> 31)) ahead += it.y; }
+            if (a >= 0) {
+                // in-block validation: the payment must fit the finalized balance minus what the
+                // payer already spent in this block (earlier batches, earlier requests of this batch)
+                const size_t ox = size_t(r) * n.N + n.origin[x];
+                const uint2* mine = n.fifo_list + size_t(r) * n.max_batch * 7 + n.in_off[ox];
+                const uint32_t mlen = n.in_deg[ox];
+                long long spent = n.blk_spent[ox];
+                for (uint32_t j = 0; j < mlen; ++j) { const uint2 it = mine[j]; if (it.x < idx && (it.y >> 31)) spent += it.y & 0x7fffffffu; }
+                const uint32_t oc = n.outcome[x];
+                const long long pay = n.R * ((oc >= 1 && oc <= 3) ? 2 : 1);
+                uncovered = n.credit[ox] - spent < pay;
+            }
             const uint64_t work = uint64_t(n.len_in[x]) + n.len_out[x], cap = n.cap_eff[px];
             const uint64_t t = (uint64_t(n.backlog[px]) + ahead + work) * 1000ull, tq = udiv64by32(t, uint32_t(cap));
             const uint64_t lat = tq + (tq * cap != t ? 1 : 0) + (a >= 0 ? n.hop_ms : 0);
@@ -267,16 +280,16 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
             lat_sum = lat; met = lat <= deadline;
         }
     }
-    const uint32_t m = __reduce_add_sync(kFull, met);
+    const uint32_t m = __reduce_add_sync(kFull, met), unc = __reduce_add_sync(kFull, uncovered);
     for (int o = 16; o; o >>= 1) lat_sum += __shfl_down_sync(kFull, lat_sum, o);
-    if ((threadIdx.x & 31) == 0) { stats_add(bs, sSloMet, m); stats_add(bs, sSumLat, lat_sum); }
+    if ((threadIdx.x & 31) == 0) { stats_add(bs, sSloMet, m); stats_add(bs, sSumLat, lat_sum); stats_add(bs, sUncovered, unc); }
     stats_end(n, bs, r);
 }
 
 void launch_fifo(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
     launch_scan_in_degrees(n, c, kFifo);
-    { Timed t(c, kFifo); k_fifo_fill<<<dim3((count * 6 + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, count); }
+    { Timed t(c, kFifo); k_fifo_fill<<<dim3((count * 7 + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, count); }
     { Timed t(c, kFifo); k_fifo_latency<<<dim3((count + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, first, count); }
 }
 

@@ -106,11 +106,11 @@ struct SettleAcc {
 
 // With exact intra-batch queueing (flag 16) the latency of a request depends on the work that
 // earlier requests of the batch put on its executor, so settle_one only records the batch's work
-// items (slot = request*6 + role: primary, challenger, four judges) and counts them per peer;
+// items (slot = request*7 + role: primary, challenger, four judges, and the origin's payment) and counts them per peer;
 // k_fifo_latency computes the latencies once the per-peer lists are built.
 __device__ __forceinline__ void fifo_emit(const Net& n, uint32_t r, uint32_t bidx, uint32_t role, int peer, uint32_t tokens)
 {
-    n.fifo_items[(size_t(r) * n.max_batch + bidx) * 6 + role] = make_int2(peer, int(tokens));
+    n.fifo_items[(size_t(r) * n.max_batch + bidx) * 7 + role] = make_int2(peer, int(tokens));
     if (peer >= 0) atomicAdd(&n.in_deg[size_t(r) * n.N + peer], 1u);
 }
 
@@ -123,6 +123,9 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
         fifo_emit(n, r, bidx, 1, duel ? b : -1, li + lo);
 #pragma unroll
         for (int l = 0; l < 4; ++l) fifo_emit(n, r, bidx, 2 + l, duel ? jd[l] : -1, li + 2u * lo);
+        const uint32_t pay = uint32_t(n.R) * (duel ? 2u : 1u);
+        fifo_emit(n, r, bidx, 6, a >= 0 ? int(o) : -1, pay);
+        if (a >= 0) add64(&n.d_spent[size_t(r) * n.N + o], (long long)pay);
     }
     const size_t base = size_t(r) * n.N;
     const uint64_t work = uint64_t(li) + lo;

@@ -16,7 +16,7 @@ enum : uint32_t { kOrigin = 1, kDraw = 2, kProbe = 3, kJudge = 4, kGossip = 5, k
 // Per-replica counters, in the order of wwws_stats_t.
 enum : uint32_t { sRequests, sLocal, sFallback, sDropped, sFailed, sDelegated, sDuel, sDuelCancelled, sDraw,
                   sJudgeEvals, sProbes, sNear, sSloMet, sSumLat, sOfflineMarks, sRounds, sBlocks, sCreditTotal,
-                  sChainHead, sPendingDigest, sCount };
+                  sChainHead, sPendingDigest, sUncovered, sCount };
 
 // Device error word codes (subset of wwws_status).
 enum : uint32_t { eArg = 1, eRange = 4, eInvariant = 6 };
@@ -52,9 +52,11 @@ struct Net {
     uint64_t* self_entry; int32_t* partner;     // partner is [Rp][N][4]
     // reverse lists of the pairwise exchange: in-degree, list offset, fill cursor, puller ids [Rp][4N]
     uint32_t* in_deg; uint32_t* in_off; uint32_t* in_cursor; int32_t* pullers;
-    // exact intra-batch queueing: work items (peer, tokens) of the batch [Rp][6*max_batch] (slot = request*6 + role)
+    // exact intra-batch queueing: work items (peer, tokens) of the batch [Rp][7*max_batch] (slot = request*7 + role; role 6 = the payment)
     // and, per peer, the list (request, tokens) of the items queued on it
     int2* fifo_items; uint2* fifo_list;
+    // credits spent since the last finalization (earlier batches of the block / this batch), for in-block validation
+    long long* blk_spent; long long* d_spent;
     // dispatch -> duel continuation, [Rp][max_batch]
     uint2* cont; uint32_t max_batch;
     const uint32_t* rank_cdf;

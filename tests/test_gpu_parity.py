@@ -203,6 +203,9 @@ def test_edge_cases_match_oracle():
     # greedy rule, with ties (equal stakes) and refusals
     cases.append(make_net(70, n_requests=400, seed=9, origin=rng.integers(0, 70, 400), flags=3 | 4, p_duel_ppm=400_000,
                           peers={"accept_ppm": 600_000, "stake_pm": rng.integers(1, 4, 70) * 300}))
+    # exact queueing + in-block validation with a payer that runs out of covered credit
+    cases.append(make_net(6, n_requests=300, seed=11, flags=3 | 16, p_duel_ppm=400_000, n_judges=2,
+                          peers=requester_first(6, credit0=np.array([5_000, 10 ** 6, 10 ** 6, 10 ** 6, 10 ** 6, 10 ** 6]))))
     for ci, (st, pa, rq) in enumerate(cases):
         g = Network(st, pa, 128); g.bind_requests(rq)
         o = Oracle(st, pa); o.bind_requests(rq)

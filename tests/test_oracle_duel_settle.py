@@ -326,3 +326,32 @@ def test_fifo_queueing_inside_a_batch_hand_cases():
                 queued[j] += 600 + 2 * 400
     assert o3.stats_dict()["sum_latency_ms"] == total
     assert np.array_equal(o3.table("backlog")[0], queued)
+
+
+def test_in_block_validation_counts_uncovered_payments():
+    """Flag 16: a payment is covered by the finalized balance minus what the payer already spent
+    in the open block (this batch and earlier batches); earnings of the open block do not count."""
+    # origin has 350 credits, R = 100: payments 1-3 are covered, 4-6 are not
+    st, pa, rq = make_net(2, n_requests=12, p_duel_ppm=0, flags=16,
+                          peers=requester_first(2, credit0=np.array([350, 10 ** 6])))
+    o = Oracle(st, pa); o.bind_requests(rq)
+    o.dispatch_batch(0, 6); o.duel_judge(); o.settle_credits(False)
+    assert o.stats_dict()["n_delegated"] == 6 and o.stats_dict()["n_uncovered"] == 3
+    # same block, next batch: the finalized balance is still 350 and 600 are already spent
+    o.dispatch_batch(6, 2); o.duel_judge(); o.settle_credits(True)
+    assert o.stats_dict()["n_uncovered"] == 5
+    # after the block is finalized the balance is 350 - 800 < R: the origin cannot delegate at all
+    o.dispatch_batch(8, 2); o.duel_judge(); o.settle_credits(True)
+    assert o.stats_dict()["n_delegated"] == 8 and o.stats_dict()["n_uncovered"] == 5
+    # a duel costs the origin 2R; earnings inside the block are not spendable
+    st2, pa2, rq2 = make_net(4, n_requests=4, p_duel_ppm=1_000_000, n_judges=1, flags=16,
+                             peers=requester_first(4, credit0=np.array([350, 10 ** 6, 10 ** 6, 10 ** 6])))
+    o2 = Oracle(st2, pa2); o2.bind_requests(rq2)
+    o2.dispatch_batch(0, 4); o2.duel_judge(); o2.settle_credits(True)
+    assert np.all(np.isin(o2.results()["outcome"][0], (1, 2)))
+    assert o2.stats_dict()["n_uncovered"] == 3              # 200 covered, then 150 left < 200 three times
+    # without the flag nothing is counted
+    st.flags = 0
+    o3 = Oracle(st, pa); o3.bind_requests(rq)
+    o3.dispatch_batch(0, 6); o3.duel_judge(); o3.settle_credits(True)
+    assert o3.stats_dict()["n_uncovered"] == 0
