@@ -350,6 +350,13 @@ def test_in_block_validation_counts_uncovered_payments():
     o2.dispatch_batch(0, 4); o2.duel_judge(); o2.settle_credits(True)
     assert np.all(np.isin(o2.results()["outcome"][0], (1, 2)))
     assert o2.stats_dict()["n_uncovered"] == 3              # 200 covered, then 150 left < 200 three times
+    # finalization closes the block: what was spent in it no longer counts against the new balance
+    st4, pa4, rq4 = make_net(2, n_requests=9, p_duel_ppm=0, flags=16,
+                             peers=requester_first(2, credit0=np.array([1000, 10 ** 6])))
+    o4 = Oracle(st4, pa4); o4.bind_requests(rq4)
+    o4.dispatch_batch(0, 6); o4.duel_judge(); o4.settle_credits(True)      # 600 spent, all covered, balance 400
+    o4.dispatch_batch(6, 3); o4.duel_judge(); o4.settle_credits(True)      # 300 more: covered by the 400
+    assert o4.stats_dict()["n_delegated"] == 9 and o4.stats_dict()["n_uncovered"] == 0
     # without the flag nothing is counted
     st.flags = 0
     o3 = Oracle(st, pa); o3.bind_requests(rq)

@@ -205,6 +205,10 @@ def test_push_pull_exchange_is_symmetric_and_faster():
             new = o.view()[0]
             ver_true = o.table("ver")[0].astype(np.uint64)
             assert np.all(new >= old) and np.all(entry_ver(new) <= ver_true[None, :])
+            # one hop per round in both modes: the version a node issued this round is known to itself
+            # and to the (at most k) partners it greeted; a pushed row is the OLD row of the pusher
+            fresh = (entry_ver(new) == ver_true[None, :]).sum(axis=0)
+            assert np.all(fresh >= 1) and np.all(fresh <= 1 + k)
             if flags == 8:
                 # somebody's old row is dominated by row i: its partner's; and row i's old content
                 # reached that partner: new[p] >= old[i] for at least one p != i
