@@ -1,6 +1,6 @@
 """Full-size parity in the benchmark's launch configuration.
 
-The three large configurations are run at their full sizes through `wwws_step` (the call the
+All five configurations are run at their full sizes through `wwws_step` (the call the
 benchmark times).  Replicas are independent and keyed by their global index, so one replica
 of the full run can be checked completely against the oracle run on that replica alone:
 every result record, every per-peer table, the counters, and sampled rows of its view matrix.
@@ -15,7 +15,8 @@ from tests.helpers import TABLE_NAMES
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,replica,steps", [("zipf1k", 200, 8), ("churn4k", 37, 12), ("adversarial16k", 5, 12)])
+@pytest.mark.parametrize("name,replica,steps", [("tiny", 0, 20), ("tiers64", 0, 200), ("zipf1k", 200, 8), ("churn4k", 37, 12),
+                                                ("adversarial16k", 5, 12)])
 def test_one_replica_of_the_full_run_matches_the_oracle(name, replica, steps):
     from paper_2603_20661_b200.binding import Network
     wl = synth.make_workload(name)
@@ -38,7 +39,8 @@ def test_one_replica_of_the_full_run_matches_the_oracle(name, replica, steps):
     assert np.array_equal(g.stats()[replica], o.stats()[0]), f"{name}: counters differ"
     ov = o.view()[0]
     N = st.n_peers
-    rows = sorted(set([0, 1, 31, 32, N // 2, N - 33, N - 1] + list(np.random.default_rng(1).integers(0, N, 40))))
+    rows = sorted(set([0, 1, min(31, N - 1), min(32, N - 1), N // 2, max(N - 33, 0), N - 1]
+                      + list(np.random.default_rng(1).integers(0, N, 40))))
     for i in rows:
         assert np.array_equal(g.view_rows(replica, int(i), 1)[0], ov[i]), f"{name}: view row {i} differs"
     # properties that hold at any size, over all replicas
