@@ -202,6 +202,13 @@ def run_gpu(args):
         roof_merge["bytes_per_launch_without_reuse"] = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
     roof_req = roof("k_step_fused", req_bytes / max(1, prof.get("k_step_fused", (0, 1))[1]))
     roofline = roof_merge if dom == "k_gossip_merge" else roof_req
+    # the whole timed region A against HBM: algorithmic bytes of its gossip rounds and requests over its duration
+    g_a, req_a = algorithmic_bytes(wl, delta)
+    rounds_a = delta["rounds"] // Rp
+    step_bytes = g_a * rounds_a + req_a
+    whole = {"bound": "hbm", "achieved": step_bytes / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+             "frac": step_bytes / (ms * 1e-3) / 1e9 / peak, "bytes_per_step": step_bytes / K,
+             "what": "all kernels of the K timed steps (gossip at its cadence + dispatch + duel + settle), algorithmic bytes"}
     # requests/s of dispatch+duel+settle alone (advance, fused step, fold, block commit), from the same events
     t_req = sum(prof[k][0] for k in ("k_advance", "k_step_fused", "k_fold", "k_finalize_check", "k_fifo") if k in prof)
     req_only = {"value": delta_b["n_requests"] / (t_req * 1e-3), "unit": UNIT, "ms_per_step": t_req / K,
@@ -250,6 +257,7 @@ def run_gpu(args):
             "roofline": roofline,
             "roofline_request_path": roof_req,
             "dispatch_duel_settle_only": req_only,
+            "whole_step_roofline": whole,
             "roofline_gossip_merge": roof_merge,
             "kernels": kernels,
             "step_mix": {k: delta[k] for k in ("n_requests", "n_delegated", "n_duel", "n_probes", "rounds")},
