@@ -3,6 +3,8 @@
 Views, ledgers, queues, executor choices, duel pairings, judge panels, outcomes and
 counters must be identical; fp32 scores within 1e-5 relative.
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -178,6 +180,50 @@ def test_fifo_queueing_matches_oracle(name, kw):
     assert_same_state(g2, o, "fifo six-call end", upto=wl.n_requests)
     base = synth.make_workload(name, **kw)
     assert o.stats_dict()["sum_latency_ms"] > 0
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("WWWS_FUZZ_SEEDS", "12"))))
+def test_random_configurations_match_oracle(seed):
+    """Seeded random small networks: sizes, fanout, judges, probe budget, probabilities, all
+    combinations of the behaviour flags, skewed ranks, misreporting, churn, stale initial views;
+    alternating call paths; everything compared after every step."""
+    from paper_2603_20661_b200.binding import Network
+    rng = np.random.default_rng(1000 + seed)
+    N = int(rng.choice([2, 3, 9, 31, 32, 33, 64, 97, 200, 513]))
+    Rp = int(rng.integers(1, 4))
+    Q, B = 360, int(rng.choice([1, 7, 60, 120]))
+    n_blk = (N + 31) // 32
+    kw = dict(fanout_k=int(rng.integers(1, 5)), gossip_tries=int(rng.integers(1, 9)), max_probes=int(rng.integers(1, 8)),
+              n_judges=int(rng.integers(1, 5)), p_duel_ppm=int(rng.choice([0, 100_000, 1_000_000])),
+              p_noise_ppm=int(rng.choice([0, 250_000])), p_leave_ppm=int(rng.choice([0, 150_000])),
+              p_join_ppm=int(rng.choice([0, 400_000])), hop_ms=int(rng.integers(0, 50)),
+              init_stale_max=int(rng.integers(0, 8)), flags=int(rng.integers(0, 32)),
+              util_window_ms=int(rng.choice([1000, 10_000])), slo_num=int(rng.integers(1, 4)), slo_den=int(rng.integers(1, 3)),
+              reward_R=int(rng.integers(1, 200)), reward_add=int(rng.integers(1, 50)), penalty_P=int(rng.integers(50, 120)))
+    if rng.random() < 0.5:
+        kw["rank_cdf"] = synth.zipf_rank_cdf(int(rng.integers(1, n_blk + 2)), 1.1)
+    shape = (Rp, N)
+    peers = {"cap_true_tok_s": rng.integers(0, 9000, shape) * (rng.random(shape) > 0.05),
+             "quality_fx": rng.integers(0, 2 ** 32, shape, dtype=np.uint64), "credit0": rng.integers(0, 3000, shape),
+             "stake_pm": rng.integers(0, 1001, shape), "offload_util_pm": rng.choice([0, 300, 700, 1001], shape),
+             "accept_util_pm": rng.choice([0, 500, 900, 1001], shape), "offload_ppm": rng.integers(0, 1_000_001, shape),
+             "accept_ppm": rng.integers(0, 1_000_001, shape), "misreport_mul": rng.integers(1, 5, shape),
+             "prio_flag": rng.integers(0, 2, shape), "online0": (rng.random(shape) > 0.1).astype(np.uint8)}
+    st, pa, rq = make_net(N, Rp, Q, seed=seed, peers=peers, origin=rng.integers(0, N, (Rp, Q)), **kw)
+    rq["len_in"] = rng.integers(1, 8193, (Rp, Q)).astype(np.uint16)
+    rq["len_out"] = rng.integers(1, 8193, (Rp, Q)).astype(np.uint16)
+    g = Network(st, pa, B); g.bind_requests(rq)
+    o = Oracle(st, pa); o.bind_requests(rq)
+    assert_same_state(g, o, f"seed {seed} create")
+    first, step = 0, 0
+    while first < Q and step < 40:
+        cnt = min(B, Q - first)
+        args = (first, cnt, 900 * (step + 1), step % 2 == 0, step % 3 != 2)
+        (g.step if step % 2 else g.run_step)(*args)
+        o.run_step(*args)
+        assert_same_state(g, o, f"seed {seed} step {step} (N={N}, flags={kw['flags']})", upto=first + cnt)
+        first += cnt; step += 1
+    g.close()
 
 
 def test_edge_cases_match_oracle():
