@@ -249,7 +249,9 @@ def run_gpu(args):
             "config": {"workload": args.workload, "n_peers": st.n_peers, "n_replicas_per_gpu": Rp,
                        "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "flags": st.flags, "gossip_every": wl.gossip_every,
                        "fanout_k": st.fanout_k, "entry": "wwws_step (fused dispatch+duel+settle)",
-                       "l2": "inputs larger than L2 (view buffers %.1f GB per GPU)" % (2 * 8 * st.n_peers ** 2 * Rp / 1e9)},
+                       "l2": ("inputs larger than L2 (view buffers %.1f GB per GPU)" % (2 * 8 * st.n_peers ** 2 * Rp / 1e9)
+                              if 2 * 8 * st.n_peers ** 2 * Rp > 126e6 else
+                              "inputs smaller than L2 and not flushed: this workload is a launch-latency case, not a bandwidth one")},
             "clocks": clocks,
             "e2e": {"value": req_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / K, "entry": "wwws_step_host, pinned host buffers"},

@@ -1,0 +1,43 @@
+"""The benchmark's reference arm (the CPU oracle timed on the host) runs without a GPU and
+prints the contract's JSON line; its helpers agree with the workload's step structure."""
+import json
+import os
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_reference_arm_prints_one_json_line():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiers64",
+                          "--steps", "6", "--warmup", "3"], capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["unit"] == "requests/s" and d["higher_is_better"] is True
+    assert d["value"] > 0 and d["steps"] == 6 and d["warmup"] == 3 and d["vs_baseline"] is None
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1
+    assert d["e2e"] == {"value": d["value"], "unit": "requests/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert d["config"]["workload"] == "tiers64"
+
+
+def test_reference_arm_other_ranks_exit_quietly():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--gpus", "2"], capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_step_schedule_and_byte_model():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2603_20661_b200 import synth
+    wl = synth.make_workload("tiny")
+    n = wl.n_steps
+    first, cnt, now, gossip = bench.step_args(wl, 0)
+    assert (first, cnt, gossip) == (0, wl.batch, True) and now == wl.step_now_ms(0)
+    f2, c2, now2, _ = bench.step_args(wl, n)             # second pass over the stream: time keeps growing
+    assert (f2, c2) == (0, wl.batch) and now2 > bench.step_args(wl, n - 1)[2]
+    g, r = bench.algorithmic_bytes(wl, {"n_requests": 10, "n_delegated": 4, "n_fallback_local": 1, "n_failed": 0})
+    assert g == 2 * 8 * 8 * 8 and r == 10 * 34 + 5 * 256
