@@ -67,8 +67,23 @@ __global__ void k_advance(Net n, uint32_t dt_ms, uint32_t now_ms)
     n.cap_eff[x] = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, now_ms);
 }
 
+// Commit of replica r's block, run by the last block of k_fold to finish that replica: total
+// credit must be what it was at creation; the chain head takes the block's operations digest.
+__device__ void finalize_replica(const Net& n, uint32_t r)
+{
+    const long long total = (long long)atomicAdd((unsigned long long*)&n.credit_check[r], 0ull);
+    if (total != n.credit_total0[r]) set_error(n, eInvariant, r);
+    n.credit_check[r] = 0;
+    unsigned long long* st = n.stats + size_t(r) * sCount;
+    st[sBlocks] += 1;
+    // block id = hash of (parent id, order-independent digest of the block's records, height)
+    st[sChainHead] = mix64(mix64(st[sChainHead] ^ chain_key(n, r)) + st[sPendingDigest] + kGamma * st[sBlocks]);
+    st[sPendingDigest] = 0;
+}
+
 // End of a settlement: queues take the batch's work; with `finalize` the pending block is
-// folded into the ledger, stakes and derived weights are refreshed and credit is summed.
+// folded into the ledger, stakes and derived weights are refreshed, credit is summed and the
+// replica's block is committed.
 __global__ void k_fold(Net n, int finalize)
 {
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -96,20 +111,16 @@ __global__ void k_fold(Net n, int finalize)
     if (finalize) {
         for (int o = 16; o; o >>= 1) csum += __shfl_down_sync(0xffffffffu, csum, o);
         if ((threadIdx.x & 31) == 0 && csum) atomicAdd((unsigned long long*)&n.credit_check[r], (unsigned long long)csum);
+        // the block that finishes a replica last commits it (no second launch): every block makes
+        // its sums visible, then takes a ticket
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0 && atomicAdd(&n.fold_ticket[r], 1u) == gridDim.x - 1) {
+            n.fold_ticket[r] = 0;
+            __threadfence();
+            finalize_replica(n, r);
+        }
     }
-}
-
-__global__ void k_finalize_check(Net n)
-{
-    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= n.Rp) return;
-    if (n.credit_check[r] != n.credit_total0[r]) set_error(n, eInvariant, r);
-    n.credit_check[r] = 0;
-    unsigned long long* st = n.stats + size_t(r) * sCount;
-    st[sBlocks] += 1;
-    // block id = hash of (parent id, order-independent digest of the block's records, height)
-    st[sChainHead] = mix64(mix64(st[sChainHead] ^ chain_key(n, r)) + st[sPendingDigest] + kGamma * st[sBlocks]);
-    st[sPendingDigest] = 0;
 }
 
 // Re-derive stake and weight from the ledger as it stands (after a table import).
@@ -158,8 +169,8 @@ void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchC
 
 void launch_fold(const Net& n, int finalize, const LaunchCtx& c)
 {
-    { Timed t(c, kFold); k_fold<<<peer_grid(n), 256, 0, c.stream>>>(n, finalize); }
-    if (finalize) { Timed t(c, kFinalizeCheck); k_finalize_check<<<(n.Rp + 127) / 128, 128, 0, c.stream>>>(n); }
+    Timed t(c, kFold);
+    k_fold<<<peer_grid(n), 256, 0, c.stream>>>(n, finalize);
 }
 
 void launch_rederive(const Net& n, const LaunchCtx& c)

@@ -62,6 +62,7 @@ struct Net {
     const uint32_t* rank_cdf;
     unsigned long long* stats;                   // [Rp][sCount]
     const int64_t* credit_total0; long long* credit_check;   // [Rp]
+    uint32_t* fold_ticket;                       // [Rp] blocks of k_fold that have finished the replica
     uint32_t* err;                               // [2]: code, detail
     // bound requests / results
     const uint32_t* origin; const uint16_t* len_in; const uint16_t* len_out; uint64_t Q;

@@ -7,7 +7,7 @@
 namespace wwws {
 
 // Kernel classes, for launch counts and optional event timing.
-enum KernelId : int { kPeerInit, kViewInit, kAdvance, kFold, kFinalizeCheck, kRederive, kCreditTotal, kGossipPeer,
+enum KernelId : int { kPeerInit, kViewInit, kAdvance, kFold, kRederive, kCreditTotal, kGossipPeer,
                       kGossipMerge, kGossipFixup, kGossipLists, kFifo, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
 
 // When enabled, every launch is bracketed by two events on the launching stream; read()

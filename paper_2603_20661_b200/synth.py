@@ -228,6 +228,59 @@ def make_workload(name: str, *, seed: int = 0, n_replicas: Optional[int] = None,
     return wl
 
 
+# Request schedules shaped like the paper's Table of experimental settings: per node
+# (relative capacity, [(interval end in s, mean inter-arrival time in s), ...]) over 750 s.
+# Only the schedule shapes are taken from the table; capacities are relative service rates
+# chosen here (the table names models and GPUs, not token rates).
+PAPER_SETTINGS = {
+    "setting1": [(1.0, [(300, 5), (750, 20)]), (1.0, [(750, 20)]), (1.0, [(750, 20)]), (1.0, [(450, 20), (750, 5)])],
+    "setting2": [(1.0, [(300, 4), (750, 20)]), (1.0, [(750, 20)]), (0.7, [(750, 30)]), (0.7, [(450, 30), (750, 6)])],
+    "setting3": [(4.0, [(300, 2), (750, 6)]), (1.0, [(750, 15)]), (0.7, [(750, 30)]), (1.0, [(450, 15), (750, 5)])],
+    "setting4": [(1.0, [(750, 9)]), (1.0, [(450, 6), (750, 12)]), (1.0, [(300, 6), (750, 12)]), (1.0, [(450, 12), (750, 6)]),
+                 (0.8, [(750, 12)]), (0.8, [(450, 10), (750, 20)]), (0.7, [(300, 20), (750, 10)]), (0.7, [(300, 20), (750, 10)])],
+}
+
+
+def make_paper_setting(name: str, *, seed: int = 0, n_replicas: int = 64, offload: bool = True,
+                       base_capacity: int = 1000, batch: int = 8) -> Workload:
+    """A small network with piecewise-Poisson per-node arrivals (hot and idle phases that differ
+    across nodes), long generations (median 6,000 output tokens, capped at 8,192 like the paper's
+    runs) and the paper's standard policy; `offload=False` gives the single-node baseline in
+    which every node serves only its own users.  All replicas share the arrival stream and differ
+    in request lengths and in the protocol's random draws."""
+    nodes = PAPER_SETTINGS[name]
+    rng = np.random.default_rng(np.random.PCG64(seed))
+    times, origins = [], []
+    for node, (_, schedule) in enumerate(nodes):
+        t, start = 0.0, 0.0
+        for end, gap in schedule:
+            t = max(t, start)
+            while True:
+                t += rng.exponential(gap)
+                if t >= end:
+                    break
+                times.append(t); origins.append(node)
+            start = end
+    order = np.argsort(np.array(times), kind="stable")
+    t_ms = np.floor(np.array(times)[order] * 1000.0).astype(np.uint32)
+    origin = np.array(origins, np.uint32)[order]
+    N, Q = len(nodes), len(order)
+    shape = (n_replicas, N)
+    st = Settings(N, n_replicas, seed=seed, fanout_k=2, p_duel_ppm=50_000, n_judges=2, cap_ref_tok_s=base_capacity,
+                  flags=3 | 16)
+    cap = np.array([int(round(c * base_capacity)) for c, _ in nodes], np.uint32)
+    peers = default_peers(rng, n_replicas, N, offload_util_pm=700)
+    peers["cap_true_tok_s"] = np.ascontiguousarray(np.broadcast_to(cap, shape))
+    if not offload:
+        peers["offload_ppm"] = np.zeros(shape, np.uint32)
+    rshape = (n_replicas, Q)
+    requests = {"origin": np.ascontiguousarray(np.broadcast_to(origin, rshape)),
+                "t_ms": np.ascontiguousarray(np.broadcast_to(t_ms, rshape)),
+                "len_in": np.clip(np.rint(np.exp(rng.normal(math.log(300.0), 0.5, rshape))), 1, 8192).astype(np.uint16),
+                "len_out": np.clip(np.rint(np.exp(rng.normal(math.log(6000.0), 0.5, rshape))), 1, 8192).astype(np.uint16)}
+    return Workload(name, st, peers, requests, batch=batch, gossip_every=1)
+
+
 def slice_replicas(wl: Workload, r0: int, r1: int) -> Workload:
     """The same workload restricted to replicas [r0, r1); randomness stays keyed
     by the global replica index through `replica_offset`."""
