@@ -170,6 +170,15 @@ def run_gpu(args):
     total_requests = int(reduce_sum_vec(np.array([delta["n_requests"]], np.uint64))[0])
     value = total_requests / (ms * 1e-3)
 
+    # a second, identical timed region: reported beside the first one so that a disturbed run shows
+    barrier()
+    ev0.record()
+    for _ in range(K):
+        net.step(*step_args(wl, s)); s += 1
+    ev1.record()
+    barrier()
+    ms_repeat = reduce_max(ev0.elapsed_time(ev1))
+
     # ---- region B: same K steps with per-kernel events (roofline of the dominant kernel) ---
     net.profile(True)
     stats_b0 = net.stats()[-1].copy()
@@ -214,6 +223,21 @@ def run_gpu(args):
     req_only = {"value": delta_b["n_requests"] / (t_req * 1e-3), "unit": UNIT, "ms_per_step": t_req / K,
                 "kernels": "k_advance + k_step_fused + k_fold (block commit included), summed CUDA-event time"}
 
+    # ---- region S: the same K steps through the six separate calls ------------------------------
+    while s % wl.gossip_every:
+        net.step(*step_args(wl, s)); s += 1
+    stats_s0 = net.stats()[-1].copy()
+    barrier()
+    ev0.record()
+    for _ in range(K):
+        net.run_step(*step_args(wl, s)); s += 1
+    ev1.record()
+    barrier()
+    ms_six = reduce_max(ev0.elapsed_time(ev1))
+    req_six = int(reduce_sum_vec(np.array([int(net.stats()[-1][0]) - int(stats_s0[0])], np.uint64))[0])
+    six = {"value": req_six / (ms_six * 1e-3), "unit": UNIT, "ms_per_step": ms_six / K,
+           "entry": "wwws_advance_time, wwws_gossip_round, wwws_dispatch_batch, wwws_duel_judge, wwws_settle_credits"}
+
     # ---- region C: end to end through host buffers ---------------------------------------------
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
     Q = wl.n_requests
@@ -244,7 +268,7 @@ def run_gpu(args):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms / K, "ms_per_step_repeat": ms_repeat / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u64 views, i64 ledgers, fp32 scores", "data": "synthetic",
             "config": {"workload": args.workload, "n_peers": st.n_peers, "n_replicas_per_gpu": Rp,
                        "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "flags": st.flags, "gossip_every": wl.gossip_every,
@@ -259,6 +283,7 @@ def run_gpu(args):
             "roofline": roofline,
             "roofline_request_path": roof_req,
             "dispatch_duel_settle_only": req_only,
+            "six_separate_calls": six,
             "whole_step_roofline": whole,
             "roofline_gossip_merge": roof_merge,
             "kernels": kernels,

@@ -252,6 +252,14 @@ wwws_status wwws_export_clock(wwws_network* net, uint32_t* now_ms, uint32_t* rou
 wwws_status wwws_import_clock(wwws_network* net, uint32_t now_ms, uint32_t round);
 wwws_status wwws_import_stats(wwws_network* net, const wwws_stats_t* host_src);
 
+/* Tuning options; results never depend on them. */
+typedef enum {
+    WWWS_OPT_REQUEST_KERNEL = 0 /* implementation of wwws_dispatch_batch / wwws_duel_judge: 0 chosen by launch size
+                                   (default), 1 one warp per request (lane per candidate, warp-shuffle prefix sums),
+                                   2 one thread per request (weights in shared memory, duels compacted per block) */
+} wwws_option;
+wwws_status wwws_set_option(wwws_network* net, wwws_option option, int64_t value);
+
 /* Kernels launched so far on behalf of this network. */
 uint64_t wwws_kernel_launches(const wwws_network* net);
 

@@ -30,7 +30,7 @@ EXPORTS = ("wwws_workspace_bytes", "wwws_create_network", "wwws_destroy_network"
            "wwws_step", "wwws_step_host", "wwws_stats", "wwws_export_table", "wwws_import_table",
            "wwws_export_view_rows", "wwws_kernel_launches", "wwws_last_error", "wwws_profile", "wwws_profile_read",
            "wwws_profile_kernels", "wwws_profile_kernel_name", "wwws_gossip_round_static", "wwws_import_view_rows",
-           "wwws_export_clock", "wwws_import_clock", "wwws_import_stats")
+           "wwws_export_clock", "wwws_import_clock", "wwws_import_stats", "wwws_set_option")
 
 
 class WwwsError(RuntimeError):
@@ -95,7 +95,7 @@ def load():
             "wwws_export_view_rows": [vp, u32, u32, u32, vp],
             "wwws_profile": [vp, i32], "wwws_profile_read": [vp, vp, vp],
             "wwws_import_view_rows": [vp, u32, u32, u32, vp], "wwws_export_clock": [vp, C.POINTER(u32), C.POINTER(u32)],
-            "wwws_import_clock": [vp, u32, u32], "wwws_import_stats": [vp, vp],
+            "wwws_import_clock": [vp, u32, u32], "wwws_import_stats": [vp, vp], "wwws_set_option": [vp, i32, C.c_int64],
         }
         for name, args in sig.items():
             f = getattr(L, name); f.argtypes = args; f.restype = C.c_int
@@ -309,6 +309,10 @@ class Network:
     def results(self):
         self._torch.cuda.synchronize(self.device)
         return {k: v.cpu().numpy() for k, v in self.res.items()}
+
+    def set_option(self, option, value):
+        """Tuning option (see wwws_option in include/wwws.h); 0 = WWWS_OPT_REQUEST_KERNEL."""
+        self._check(load().wwws_set_option(self._h, int(option), int(value)), self._h)
 
     def profile(self, enable):
         """Switch per-kernel event timing on or off (clears the sums)."""

@@ -21,6 +21,7 @@ struct wwws_network {
     int phase;                   // 0 idle, 1 dispatched, 2 judged
     uint64_t batch_first; uint32_t batch_count;
     bool bound;
+    int request_kernel;          // 0 by launch size, 1 warp per request, 2 thread per request
     uint64_t launches;
     Profiler prof;
     std::string err;
@@ -296,10 +297,21 @@ static wwws_status check_batch(wwws_network* n, uint64_t first, uint64_t count)
     return WWWS_OK;
 }
 
+// The separate dispatch and duel calls have two implementations with identical results: one warp
+// per request (lane per candidate; shortest latency, best for small batches) and one thread per
+// request (far fewer instructions per request; best from a few thousand requests per launch).
+static bool threads_for(const wwws_network* n, uint64_t count)
+{
+    if (n->request_kernel == 1) return false;
+    if (n->request_kernel == 2) return true;
+    return count * n->d.Rp >= 8192;
+}
+
 wwws_status wwws_dispatch_batch(wwws_network* n, uint64_t first, uint64_t count)
 {
     if (wwws_status st = check_batch(n, first, count)) return st;
-    launch_dispatch(n->d, first, uint32_t(count), n->ctx());
+    if (threads_for(n, count)) launch_dispatch_threads(n->d, first, uint32_t(count), n->ctx());
+    else launch_dispatch(n->d, first, uint32_t(count), n->ctx());
     n->batch_first = first; n->batch_count = uint32_t(count); n->phase = 1;
     return launch_status(n, "dispatch_batch");
 }
@@ -308,7 +320,8 @@ wwws_status wwws_duel_judge(wwws_network* n)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 1) return fail(n, WWWS_ERR_STATE, "duel_judge must follow dispatch_batch");
-    launch_duel(n->d, n->batch_first, n->batch_count, n->ctx());
+    if (threads_for(n, n->batch_count)) launch_duel_threads(n->d, n->batch_first, n->batch_count, n->ctx());
+    else launch_duel(n->d, n->batch_first, n->batch_count, n->ctx());
     n->phase = 2;
     return launch_status(n, "duel_judge");
 }
@@ -459,6 +472,19 @@ wwws_status wwws_import_stats(wwws_network* n, const wwws_stats_t* host_src)
     CUDA_TRY(n, cudaMemcpyAsync(n->d.stats, host_src, uint64_t(n->d.Rp) * sizeof(wwws_stats_t), cudaMemcpyHostToDevice, n->stream));
     CUDA_TRY(n, cudaStreamSynchronize(n->stream));
     return WWWS_OK;
+}
+
+wwws_status wwws_set_option(wwws_network* n, wwws_option option, int64_t value)
+{
+    if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    switch (option) {
+    case WWWS_OPT_REQUEST_KERNEL:
+        if (value < 0 || value > 2) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_REQUEST_KERNEL takes 0 (by size), 1 (warp) or 2 (thread)");
+        n->request_kernel = int(value);
+        return WWWS_OK;
+    default:
+        return fail(n, WWWS_ERR_ARG, "unknown option");
+    }
 }
 
 uint64_t wwws_kernel_launches(const wwws_network* n) { return n ? n->launches : 0; }

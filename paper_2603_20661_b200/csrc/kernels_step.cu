@@ -107,7 +107,44 @@ __device__ __forceinline__ int find_peer(const Net& n, StepShared<BT>& sh, uint3
     return -1;
 }
 
+// Scores the window of request (o, blk) into shared memory; returns the four group sums through d
+// and the lane-ascending fp32 sum of the scores.
 template <int BT>
+__device__ __forceinline__ float score_window(const Net& n, StepShared<BT>& sh, uint32_t slot, uint32_t r, uint32_t o, uint32_t blk,
+                                              uint32_t keep, Draws& d)
+{
+    const uint64_t* win = n.view + (size_t(r) * n.N + o) * n.ld + kWin * blk;
+    const float* wled = n.w_led + size_t(r) * n.N;
+    float ssum = 0.0f;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        uint64_t gsum = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c0 = 8 * g + 4 * h;
+            const ulonglong4 e4 = *reinterpret_cast<const ulonglong4*>(win + c0);     // 32 B of the window
+            const uint64_t e[4] = { e4.x, e4.y, e4.z, e4.w };
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t id = kWin * blk + c0 + j;
+                const float wl = id < n.N ? wled[id] : 0.0f;
+                float sc;
+                uint64_t W = candidate_weight(n, o, id, e[j], wl, sc);
+                if (!(keep >> (c0 + j) & 1u)) W = 0;                                       // lanes already drawn (duel pass)
+                sh.W[c0 + j][slot] = W;
+                gsum += W;
+                ssum = __fadd_rn(ssum, sc);                                                // lane-ascending fp32 sum
+            }
+        }
+        if (g == 0) d.G0 = gsum; else if (g == 1) d.G1 = gsum; else if (g == 2) d.G2 = gsum; else d.G3 = gsum;
+    }
+    return ssum;
+}
+
+// What a launch does: the whole step, or one of the two calls it replaces on large batches.
+enum : int { kModeFused = 0, kModeDispatch = 1, kModeDuel = 2 };
+
+template <int BT, int MODE>
 __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32_t count)
 {
     __shared__ StepShared<BT> sh;
@@ -119,74 +156,86 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
     const uint32_t idx = blockIdx.x * BT + slot;
     SettleAcc acc; acc_zero(acc);
 
-    // ---- dispatch (D1..D6), one request per thread -----------------------------------------
-    if (idx < count) {
-        const uint32_t q = uint32_t(first + idx);
-        const size_t x = size_t(r) * n.Q + first + idx;
-        const uint32_t o = n.origin[x];
-        const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
-        int a;
-        float sa = 0.0f, ssum = 0.0f;
-        Draws d;
-        d.G0 = d.G1 = d.G2 = d.G3 = 0; d.n_draws = 0; d.n_probes = 0; d.near = false; d.y_slot = 0xffffffffu;
-        uint32_t blk = 0;
-        bool duel = false;
-        if (origin_offloads(n, r, o, rx, a)) {
-            const int local_code = a;
-            blk = pick_block(n, o, rx.w[2]);
-            const uint64_t* win = n.view + (size_t(r) * n.N + o) * n.ld + kWin * blk;
-            const float* wled = n.w_led + size_t(r) * n.N;
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                uint64_t gsum = 0;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int c0 = 8 * g + 4 * h;
-                    const ulonglong4 e4 = *reinterpret_cast<const ulonglong4*>(win + c0);     // 32 B of the window
-                    const uint64_t e[4] = { e4.x, e4.y, e4.z, e4.w };
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t id = kWin * blk + c0 + j;
-                        const float wl = id < n.N ? wled[id] : 0.0f;
+    if (MODE != kModeDuel) {
+        // ---- dispatch (D1..D6), one request per thread -------------------------------------
+        if (idx < count) {
+            const uint32_t q = uint32_t(first + idx);
+            const size_t x = size_t(r) * n.Q + first + idx;
+            const uint32_t o = n.origin[x];
+            const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
+            int a;
+            float sa = 0.0f, ssum = 0.0f;
+            Draws d;
+            d.G0 = d.G1 = d.G2 = d.G3 = 0; d.n_draws = 0; d.n_probes = 0; d.near = false; d.y_slot = 0xffffffffu;
+            uint32_t blk = 0;
+            bool duel = false, scored = false;
+            if (origin_offloads(n, r, o, rx, a)) {
+                const int local_code = a;
+                blk = pick_block(n, o, rx.w[2]);
+                ssum = score_window<BT>(n, sh, slot, r, o, blk, 0xffffffffu, d);
+                scored = true;
+                a = find_peer<BT>(n, sh, slot, d, r, rg, q, blk);
+                if (a >= 0) {
+                    if (n.score_a) {
                         float sc;
-                        const uint64_t W = candidate_weight(n, o, id, e[j], wl, sc);
-                        sh.W[c0 + j][slot] = W;
-                        gsum += W;
-                        ssum = __fadd_rn(ssum, sc);                                            // lane-ascending fp32 sum
+                        candidate_weight(n, o, uint32_t(a), n.view[(size_t(r) * n.N + o) * n.ld + a], n.w_led[size_t(r) * n.N + a], sc);
+                        sa = sc;
                     }
-                }
-                if (g == 0) d.G0 = gsum; else if (g == 1) d.G1 = gsum; else if (g == 2) d.G2 = gsum; else d.G3 = gsum;
+                    duel = ppm(rx.w[1]) < n.p_duel;
+                } else a = local_code == -4 ? -4 : -2;
             }
-            a = find_peer<BT>(n, sh, slot, d, r, rg, q, blk);
-            if (a >= 0) {
-                if (n.score_a) {
-                    float sc;
-                    candidate_weight(n, o, uint32_t(a), win[a & 31], wled[a], sc);
-                    sa = sc;
+            n.exec_a[x] = a;
+            if (n.score_a) n.score_a[x] = sa;
+            if (n.score_sum) n.score_sum[x] = ssum;
+            if (MODE == kModeFused && duel) {
+                const uint32_t k = atomicAdd(&sh.n_duel, 1u);
+                sh.queue[k] = uint16_t(slot);
+                sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
+                sh.ctx[slot].draws_probes_near = d.n_draws | (d.n_probes << 8) | (d.near ? 1u << 16 : 0u);
+            } else {
+                n.exec_b[x] = -1; n.outcome[x] = 0; n.rflags[x] = d.near ? 1 : 0;
+                *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(-1, -1, -1, -1);
+                acc.c[sProbes] += d.n_probes;
+                if (MODE == kModeFused) {
+                    const int jd[4] = { -1, -1, -1, -1 };
+                    settle_one(n, r, q, idx, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
+                } else {
+                    // continuation for the duel call: lanes still in play, draws and probes used
+                    uint32_t mask = 0;
+                    if (scored) {
+#pragma unroll
+                        for (int c = 0; c < int(kWin); ++c) mask |= (sh.W[c][slot] != 0 ? 1u : 0u) << c;
+                    }
+                    n.cont[size_t(r) * n.max_batch + idx] = make_uint2(mask, d.n_draws | (d.n_probes << 8));
                 }
-                duel = ppm(rx.w[1]) < n.p_duel;
-            } else a = local_code == -4 ? -4 : -2;
+            }
         }
-        n.exec_a[x] = a;
-        if (n.score_a) n.score_a[x] = sa;
-        if (n.score_sum) n.score_sum[x] = ssum;
-        if (duel) {
-            const uint32_t k = atomicAdd(&sh.n_duel, 1u);
-            sh.queue[k] = uint16_t(slot);
-            sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
-            sh.ctx[slot].draws_probes_near = d.n_draws | (d.n_probes << 8) | (d.near ? 1u << 16 : 0u);
-        } else {
-            n.exec_b[x] = -1; n.outcome[x] = 0; n.rflags[x] = d.near ? 1 : 0;
-            *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(-1, -1, -1, -1);
-            const int jd[4] = { -1, -1, -1, -1 };
-            acc.c[sProbes] += d.n_probes;
-            settle_one(n, r, q, idx, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
+    } else {
+        // ---- duel call: requests flagged as duels re-create their window and queue up ----------
+        if (idx < count) {
+            const uint32_t q = uint32_t(first + idx);
+            const size_t x = size_t(r) * n.Q + first + idx;
+            const int a = n.exec_a[x];
+            if (a >= 0) {
+                const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
+                if (ppm(rx.w[1]) < n.p_duel) {
+                    const uint32_t o = n.origin[x];
+                    const uint2 ct = n.cont[size_t(r) * n.max_batch + idx];
+                    const uint32_t blk = pick_block(n, o, rx.w[2]);
+                    Draws d;
+                    score_window<BT>(n, sh, slot, r, o, blk, ct.x, d);
+                    const uint32_t k = atomicAdd(&sh.n_duel, 1u);
+                    sh.queue[k] = uint16_t(slot);
+                    sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
+                    sh.ctx[slot].draws_probes_near = (ct.y & 0xffffu) | ((n.rflags[x] & 1u) << 16);
+                }
+            }
         }
     }
     __syncthreads();
 
     // ---- duel-and-judge (J2, J3) for the queued requests, densely -----------------------------
-    if (threadIdx.x < sh.n_duel) {
+    if (MODE != kModeDispatch && threadIdx.x < sh.n_duel) {
         const uint32_t ds = sh.queue[threadIdx.x];
         const uint32_t didx = blockIdx.x * BT + ds;
         const uint32_t q = uint32_t(first + didx);
@@ -195,6 +244,7 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
         const uint32_t blk = sh.ctx[ds].blk, packed = sh.ctx[ds].draws_probes_near;
         Draws d;
         d.n_draws = packed & 0xffu; d.n_probes = (packed >> 8) & 0xffu; d.near = (packed >> 16) & 1u; d.y_slot = 0xffffffffu;
+        const uint32_t probes0 = d.n_probes;
         uint64_t gs[4];
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
@@ -230,10 +280,15 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
                 oc = 2 * votes_a > nj ? 1u : (2 * votes_a < nj ? 2u : 3u);
             }
         }
+        if (oc == 4) { b = -1; jd[0] = jd[1] = jd[2] = jd[3] = -1; }
         n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = d.near ? 1 : 0;
         *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
-        acc.c[sProbes] += d.n_probes;
-        settle_one(n, r, q, didx, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
+        if (MODE == kModeFused) {
+            acc.c[sProbes] += d.n_probes;
+            settle_one(n, r, q, didx, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
+        } else {
+            acc.c[sProbes] += d.n_probes - probes0;
+        }
     }
 
     // ---- counters: warp reduce, block reduce, one atomic per counter and block ---------------
@@ -251,14 +306,32 @@ __global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32
     stats_end(n, sh.stats, r);
 }
 
+template <int MODE>
+static void launch_by_size(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    // small batches: small blocks, so that the requests spread over all SMs
+    if (uint64_t(count) * n.Rp >= 148ull * 128 * 4)
+        k_step_fused<128, MODE><<<dim3((count + 127) / 128, n.Rp), 128, 0, c.stream>>>(n, first, count);
+    else
+        k_step_fused<32, MODE><<<dim3((count + 31) / 32, n.Rp), 32, 0, c.stream>>>(n, first, count);
+}
+
 void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
     Timed t(c, kStepFused);
-    // small batches: small blocks, so that the requests spread over all SMs
-    if (uint64_t(count) * n.Rp >= 148ull * 128 * 4)
-        k_step_fused<128><<<dim3((count + 127) / 128, n.Rp), 128, 0, c.stream>>>(n, first, count);
-    else
-        k_step_fused<32><<<dim3((count + 31) / 32, n.Rp), 32, 0, c.stream>>>(n, first, count);
+    launch_by_size<kModeFused>(n, first, count, c);
+}
+
+// Thread-per-request versions of the separate dispatch and duel calls (large batches).
+void launch_dispatch_threads(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    Timed t(c, kDispatch);
+    launch_by_size<kModeDispatch>(n, first, count, c);
+}
+void launch_duel_threads(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    Timed t(c, kDuel);
+    launch_by_size<kModeDuel>(n, first, count, c);
 }
 
 }  // namespace wwws

@@ -68,6 +68,31 @@ def test_six_calls_match_oracle_after_every_call(name, kw, steps):
 
 
 @pytest.mark.parametrize("name,kw,steps", CASES, ids=[c[0] for c in CASES])
+def test_six_calls_with_thread_kernels_match_oracle(name, kw, steps):
+    """The thread-per-request implementation of the separate dispatch and duel calls, forced on."""
+    wl = synth.make_workload(name, **kw)
+    g, o = _pair(wl)
+    g.set_option(0, 2)
+    for s in range(wl.n_steps):
+        first = s * wl.batch
+        cnt = min(wl.batch, wl.n_requests - first)
+        for sim in (g, o):
+            sim.advance_time(wl.step_now_ms(s))
+            if s % wl.gossip_every == 0:
+                sim.gossip_round()
+            sim.dispatch_batch(first, cnt)
+        if s < 3:
+            assert_same_state(g, o, f"step {s} dispatch", upto=first + cnt, views=False, stats=False)
+        g.duel_judge(); o.duel_judge()
+        if s < 3:
+            assert_same_state(g, o, f"step {s} duel", upto=first + cnt, views=False, stats=False)
+        g.settle_credits(s % 2 == 0); o.settle_credits(s % 2 == 0)
+        if s < 3 or s % 5 == 0:
+            assert_same_state(g, o, f"step {s} settle", upto=first + cnt, views=False)
+    assert_same_state(g, o, "end", upto=wl.n_requests)
+
+
+@pytest.mark.parametrize("name,kw,steps", CASES, ids=[c[0] for c in CASES])
 def test_fused_step_matches_oracle(name, kw, steps):
     wl = synth.make_workload(name, **kw)
     g, o = _pair(wl)
@@ -213,6 +238,7 @@ def test_random_configurations_match_oracle(seed):
     rq["len_in"] = rng.integers(1, 8193, (Rp, Q)).astype(np.uint16)
     rq["len_out"] = rng.integers(1, 8193, (Rp, Q)).astype(np.uint16)
     g = Network(st, pa, B); g.bind_requests(rq)
+    g.set_option(0, 1 + seed % 2)                # six-call path: warp-per-request / thread-per-request kernels in turn
     o = Oracle(st, pa); o.bind_requests(rq)
     assert_same_state(g, o, f"seed {seed} create")
     first, step = 0, 0
