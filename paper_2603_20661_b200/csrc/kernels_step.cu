@@ -145,7 +145,7 @@ __device__ __forceinline__ float score_window(const Net& n, StepShared<BT>& sh, 
 enum : int { kModeFused = 0, kModeDispatch = 1, kModeDuel = 2 };
 
 template <int BT, int MODE>
-__global__ void __launch_bounds__(BT) k_step_fused(Net n, uint64_t first, uint32_t count)
+__global__ void __launch_bounds__(BT, BT == 128 ? 5 : 1) k_step_fused(Net n, uint64_t first, uint32_t count)
 {
     __shared__ StepShared<BT> sh;
     stats_begin(sh.stats);                       // barrier inside
