@@ -58,6 +58,9 @@ typedef enum {
                                    judge evaluations), not only the executor's queue at the start of the batch;
                                    also validates every payment against the payer's balance inside the open block
                                    (n_uncovered) */
+#define WWWS_FLAG_MAJORITY 32u  /* a block is committed only if more than half of the peers are online to confirm it
+                                   (Section "Credit-based Transaction System"); otherwise it stays open and its
+                                   operations are committed with the next block that finds a majority */
 #define WWWS_FLAG_GREEDY 4u     /* customised rule: instead of drawing in proportion to the weights, take the
                                    candidate with the highest weight (lowest id on ties), then the next one on
                                    refusal; flags bit 0 then marks a runner-up within 1e-5 (relative) of the pick */
@@ -140,6 +143,7 @@ typedef struct {
                                 operations settled since the last finalization */
     uint64_t n_uncovered;    /* with WWWS_FLAG_FIFO: payments that exceeded the payer's finalized balance minus
                                 what it had already spent in the open block (double-spend check; counted only) */
+    uint64_t blocks_rejected;/* with WWWS_FLAG_MAJORITY: finalizations refused for want of a majority */
 } wwws_stats_t;
 
 /* Per-peer tables for wwws_export_table / wwws_import_table; element type in the comment. */

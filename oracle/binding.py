@@ -19,7 +19,7 @@ _SO = os.path.join(_HERE, "libwwws_oracle.so")
 
 STAT_NAMES = ("n_requests", "n_local", "n_fallback_local", "n_dropped", "n_failed", "n_delegated", "n_duel",
               "n_duel_cancelled", "n_draw", "n_judge_evals", "n_probes", "n_near_boundary", "slo_met",
-              "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest", "n_uncovered")
+              "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest", "n_uncovered", "blocks_rejected")
 TABLES = ("online", "cap_eff", "backlog", "ver", "credit", "stake", "wins", "duels", "served", "served_local",
           "d_credit", "d_wins", "d_duels")
 

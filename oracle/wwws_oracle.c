@@ -115,7 +115,7 @@ typedef struct {
 
 enum { S_REQUESTS, S_LOCAL, S_FALLBACK, S_DROPPED, S_FAILED, S_DELEGATED, S_DUEL, S_DUEL_CANCELLED, S_DRAW,
        S_JUDGE_EVALS, S_PROBES, S_NEAR, S_SLO_MET, S_SUM_LAT, S_OFFLINE_MARKS, S_ROUNDS, S_BLOCKS, S_CREDIT_TOTAL,
-       S_CHAIN_HEAD, S_PENDING_DIGEST, S_UNCOVERED, S_N };
+       S_CHAIN_HEAD, S_PENDING_DIGEST, S_UNCOVERED, S_BLOCKS_REJECTED, S_N };
 
 typedef struct {
     uint32_t inplay;       /* lanes still in play after the draws so far */
@@ -643,11 +643,20 @@ int orc_settle_credits(orc_net *n, int finalize)
             st[S_SUM_LAT] += lat;
             if (lat <= deadline) st[S_SLO_MET] += 1;
         }
+        /* majority validation (flag 32; Section "Credit-based Transaction System": a block is final once
+         * a majority of peers confirm and append it): every online peer validates the proposed block; without
+         * a majority the block stays open and its operations ride along with the next proposal */
+        int commit = finalize;
+        if (commit && (c->flags & 32)) {
+            uint32_t online = 0;
+            for (uint32_t j = 0; j < n->N; ++j) online += P[j].online;
+            if (2 * online <= n->N) { commit = 0; st[S_BLOCKS_REJECTED] += 1; }
+        }
         for (uint32_t j = 0; j < n->N; ++j) {
             P[j].backlog += P[j].d_backlog; P[j].d_backlog = 0;
-            P[j].blk_spent = finalize ? 0 : P[j].blk_spent + P[j].d_spent; P[j].d_spent = 0;
+            P[j].blk_spent = commit ? 0 : P[j].blk_spent + P[j].d_spent; P[j].d_spent = 0;
         }
-        if (finalize) finalize_replica(n, r);
+        if (commit) finalize_replica(n, r);
     }
     n->phase = 0;
     return 0;

@@ -20,7 +20,7 @@ STATUS = {0: "OK", 1: "ERR_ARG", 2: "ERR_ALLOC", 3: "ERR_STATE", 4: "ERR_RANGE",
           7: "ERR_TIMEOUT"}
 STAT_NAMES = ("n_requests", "n_local", "n_fallback_local", "n_dropped", "n_failed", "n_delegated", "n_duel",
               "n_duel_cancelled", "n_draw", "n_judge_evals", "n_probes", "n_near_boundary", "slo_met",
-              "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest", "n_uncovered")
+              "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest", "n_uncovered", "blocks_rejected")
 TABLES = {"online": (0, np.uint8), "cap_eff": (1, np.uint32), "backlog": (2, np.int64), "ver": (3, np.uint32),
           "credit": (4, np.int64), "stake": (5, np.int64), "wins": (6, np.uint32), "duels": (7, np.uint32),
           "served": (8, np.uint64), "served_local": (9, np.uint64), "d_credit": (10, np.int64),

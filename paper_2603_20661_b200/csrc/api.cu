@@ -114,7 +114,7 @@ void carve(const wwws_config& c, Carver& cv, Net& d, Staging& sg)
     d.rank_cdf = c.n_rank ? cv.take<uint32_t>(c.n_rank) : nullptr;
     d.stats = cv.take<unsigned long long>(Rp * sCount);
     d.credit_total0 = cv.take<int64_t>(Rp); d.credit_check = cv.take<long long>(Rp);
-    d.fold_ticket = cv.take<uint32_t>(Rp);
+    d.fold_ticket = cv.take<uint32_t>(Rp); d.online_count = cv.take<uint32_t>(Rp);
     d.err = cv.take<uint32_t>(4);
     sg.credit0 = cv.take<int64_t>(NP); sg.online0 = cv.take<uint8_t>(NP);
     cv.off = (cv.off + 255) & ~uint64_t(255);
@@ -230,6 +230,7 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
     }
     CUDA_TRY(nullptr, cudaMemsetAsync(d.credit_check, 0, d.Rp * 8ull, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.fold_ticket, 0, d.Rp * 4ull, s));
+    CUDA_TRY(nullptr, cudaMemsetAsync(d.online_count, 0, d.Rp * 4ull, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.err, 0, 16, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.partner, 0xff, NP * 16, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.in_deg, 0, NP * 4, s));

@@ -84,9 +84,20 @@ __device__ void finalize_replica(const Net& n, uint32_t r)
 // End of a settlement: queues take the batch's work; with `finalize` the pending block is
 // folded into the ledger, stakes and derived weights are refreshed, credit is summed and the
 // replica's block is committed.
-__global__ void k_fold(Net n, int finalize)
+// Majority validation: how many peers of each replica are online to confirm a proposed block.
+__global__ void k_count_online(Net n)
 {
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t on = j < n.N && n.online[size_t(r) * n.N + j];
+    const uint32_t c = __reduce_add_sync(0xffffffffu, on);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&n.online_count[r], c);
+}
+
+__global__ void k_fold(Net n, int finalize_requested)
+{
+    const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
+    // with majority validation the block is committed only if more than half of the peers are online
+    const bool finalize = finalize_requested && (!(n.flags & 32u) || 2u * n.online_count[r] > n.N);
     long long csum = 0;
     if (j < n.N) {
         const size_t x = size_t(r) * n.N + j;
@@ -120,7 +131,16 @@ __global__ void k_fold(Net n, int finalize)
             __threadfence();
             finalize_replica(n, r);
         }
+    } else if (finalize_requested && blockIdx.x == 0 && threadIdx.x == 0) {
+        n.stats[size_t(r) * sCount + sBlocksRejected] += 1;      // no majority: the block stays open
     }
+}
+
+// The online counts are consumed by one k_fold; clear them for the next proposal.
+__global__ void k_clear_online_count(Net n)
+{
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < n.Rp) n.online_count[r] = 0;
 }
 
 // Re-derive stake and weight from the ledger as it stands (after a table import).
@@ -169,8 +189,10 @@ void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchC
 
 void launch_fold(const Net& n, int finalize, const LaunchCtx& c)
 {
-    Timed t(c, kFold);
-    k_fold<<<peer_grid(n), 256, 0, c.stream>>>(n, finalize);
+    const bool majority = finalize && (n.flags & 32u);
+    if (majority) { Timed t(c, kFold); k_count_online<<<peer_grid(n), 256, 0, c.stream>>>(n); }
+    { Timed t(c, kFold); k_fold<<<peer_grid(n), 256, 0, c.stream>>>(n, finalize); }
+    if (majority) { Timed t(c, kFold); k_clear_online_count<<<(n.Rp + 127) / 128, 128, 0, c.stream>>>(n); }
 }
 
 void launch_rederive(const Net& n, const LaunchCtx& c)

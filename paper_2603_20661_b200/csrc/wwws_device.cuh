@@ -16,7 +16,7 @@ enum : uint32_t { kOrigin = 1, kDraw = 2, kProbe = 3, kJudge = 4, kGossip = 5, k
 // Per-replica counters, in the order of wwws_stats_t.
 enum : uint32_t { sRequests, sLocal, sFallback, sDropped, sFailed, sDelegated, sDuel, sDuelCancelled, sDraw,
                   sJudgeEvals, sProbes, sNear, sSloMet, sSumLat, sOfflineMarks, sRounds, sBlocks, sCreditTotal,
-                  sChainHead, sPendingDigest, sUncovered, sCount };
+                  sChainHead, sPendingDigest, sUncovered, sBlocksRejected, sCount };
 
 // Device error word codes (subset of wwws_status).
 enum : uint32_t { eArg = 1, eRange = 4, eInvariant = 6 };
@@ -62,6 +62,7 @@ struct Net {
     const uint32_t* rank_cdf;
     unsigned long long* stats;                   // [Rp][sCount]
     const int64_t* credit_total0; long long* credit_check;   // [Rp]
+    uint32_t* online_count;                      // [Rp] majority validation: peers online when a block is proposed
     uint32_t* fold_ticket;                       // [Rp] blocks of k_fold that have finished the replica
     uint32_t* err;                               // [2]: code, detail
     // bound requests / results

@@ -34,7 +34,7 @@ def test_struct_layouts_match_the_header():
     assert C.sizeof(binding.Config) == 16 + 8 + 18 * 4 + 3 * 8 + 8
     assert C.sizeof(binding.PeerInit) == 11 * 8 and C.sizeof(binding.Requests) == 32
     assert C.sizeof(binding.Results) == 7 * 8 and C.sizeof(binding.HostIO) == 8 * 8
-    assert len(binding.STAT_NAMES) == 21
+    assert len(binding.STAT_NAMES) == 22
 
 
 def test_host_side_argument_checks():

@@ -222,7 +222,7 @@ def test_random_configurations_match_oracle(seed):
               n_judges=int(rng.integers(1, 5)), p_duel_ppm=int(rng.choice([0, 100_000, 1_000_000])),
               p_noise_ppm=int(rng.choice([0, 250_000])), p_leave_ppm=int(rng.choice([0, 150_000])),
               p_join_ppm=int(rng.choice([0, 400_000])), hop_ms=int(rng.integers(0, 50)),
-              init_stale_max=int(rng.integers(0, 8)), flags=int(rng.integers(0, 32)),
+              init_stale_max=int(rng.integers(0, 8)), flags=int(rng.integers(0, 64)),
               util_window_ms=int(rng.choice([1000, 10_000])), slo_num=int(rng.integers(1, 4)), slo_den=int(rng.integers(1, 3)),
               reward_R=int(rng.integers(1, 200)), reward_add=int(rng.integers(1, 50)), penalty_P=int(rng.integers(50, 120)))
     if rng.random() < 0.5:
@@ -275,6 +275,9 @@ def test_edge_cases_match_oracle():
     # greedy rule, with ties (equal stakes) and refusals
     cases.append(make_net(70, n_requests=400, seed=9, origin=rng.integers(0, 70, 400), flags=3 | 4, p_duel_ppm=400_000,
                           peers={"accept_ppm": 600_000, "stake_pm": rng.integers(1, 4, 70) * 300}))
+    # majority validation under heavy churn: some blocks stay open
+    cases.append(make_net(31, n_requests=300, seed=12, origin=rng.integers(0, 31, 300), flags=3 | 32, p_duel_ppm=300_000,
+                          p_leave_ppm=500_000, p_join_ppm=400_000, peers={"credit0": 10 ** 5}))
     # exact queueing + in-block validation with a payer that runs out of covered credit
     cases.append(make_net(6, n_requests=300, seed=11, flags=3 | 16, p_duel_ppm=400_000, n_judges=2,
                           peers=requester_first(6, credit0=np.array([5_000, 10 ** 6, 10 ** 6, 10 ** 6, 10 ** 6, 10 ** 6]))))

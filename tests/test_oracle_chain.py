@@ -118,3 +118,45 @@ def test_chain_detects_changed_record_parent_and_height():
         assert o.stats_dict()["pending_digest"] == 0
         ids.append(o.stats_dict()["chain_head"])
     assert len(set(ids)) == 3
+
+
+def test_majority_validation_keeps_a_block_open_without_a_majority():
+    """Flag 32: a proposed block is final only if more than half of the peers are online to
+    confirm it; otherwise ledger, stakes and chain head stay as they were and the operations
+    are committed with the next block that finds a majority."""
+    from tests.helpers import make_net, requester_first
+    st, pa, rq = make_net(5, n_requests=30, seed=2, p_duel_ppm=500_000, n_judges=1, flags=32,
+                          peers=requester_first(5, credit0=10 ** 6))
+    o = Oracle(st, pa); o.bind_requests(rq)
+    o.run_step(0, 10, 0, False, True)
+    d1 = o.stats_dict(); c1 = o.table("credit").copy()
+    assert d1["blocks"] == 1 and d1["blocks_rejected"] == 0
+    for j in (2, 3, 4):                                   # three of five crash: two online, no majority
+        o.poke_peer(0, j, online=0)
+    o.run_step(10, 10, 0, False, True)
+    d2 = o.stats_dict()
+    assert d2["blocks"] == 1 and d2["blocks_rejected"] == 1 and d2["chain_head"] == d1["chain_head"]
+    assert np.array_equal(o.table("credit"), c1) and d2["pending_digest"] != 0
+    assert np.any(o.table("d_credit") != 0) and d2["credit_total"] == d1["credit_total"]
+    o.poke_peer(0, 2, online=1)                           # three online again: majority
+    o.run_step(20, 10, 0, False, True)
+    d3 = o.stats_dict()
+    assert d3["blocks"] == 2 and d3["blocks_rejected"] == 1 and d3["pending_digest"] == 0
+    assert np.all(o.table("d_credit") == 0) and o.table("credit").sum() == c1.sum()
+    # the delayed block holds the operations of both batches: same ledger as one block over both
+    st2, pa2, rq2 = make_net(5, n_requests=30, seed=2, p_duel_ppm=500_000, n_judges=1, flags=0,
+                             peers=requester_first(5, credit0=10 ** 6))
+    o2 = Oracle(st2, pa2); o2.bind_requests(rq2)
+    o2.run_step(0, 10, 0, False, True)
+    for j in (2, 3, 4):
+        o2.poke_peer(0, j, online=0)
+    o2.run_step(10, 10, 0, False, False)
+    o2.poke_peer(0, 2, online=1)
+    o2.run_step(20, 10, 0, False, True)
+    assert np.array_equal(o2.table("credit"), o.table("credit"))
+    assert o2.stats_dict()["chain_head"] == d3["chain_head"]
+    # exactly half is not a majority
+    st3, pa3, rq3 = make_net(4, n_requests=5, flags=32, p_duel_ppm=0, peers={"online0": np.array([1, 1, 0, 0])})
+    o3 = Oracle(st3, pa3); o3.bind_requests(rq3)
+    o3.run_step(0, 5, 0, False, True)
+    assert o3.stats_dict()["blocks"] == 0 and o3.stats_dict()["blocks_rejected"] == 1
