@@ -45,6 +45,23 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
     *reinterpret_cast<int4*>(n.partner + x * 4) = make_int4(part[0], part[1], part[2], part[3]);
 }
 
+// Once every peer's churn is known, a chosen partner either answers (it is online) or not.  The
+// partner list is rewritten in place so that the kernels that follow need no second lookup:
+// p >= 0 = answered, -2 - p = chosen but dead, -1 = no partner in that slot.
+__global__ void k_gossip_resolve(Net n)
+{
+    const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n.N) return;
+    const size_t x = size_t(r) * n.N + i;
+    int4 p4 = *reinterpret_cast<const int4*>(n.partner + x * 4);
+    const uint8_t* on = n.online + size_t(r) * n.N;
+    if (p4.x >= 0 && !on[p4.x]) p4.x = -2 - p4.x;
+    if (p4.y >= 0 && !on[p4.y]) p4.y = -2 - p4.y;
+    if (p4.z >= 0 && !on[p4.z]) p4.z = -2 - p4.z;
+    if (p4.w >= 0 && !on[p4.w]) p4.w = -2 - p4.w;
+    *reinterpret_cast<int4*>(n.partner + x * 4) = p4;
+}
+
 // Streaming merge: new row = max(old row, rows of the partners that answered).
 //
 // A row is read by its owner and by every node that pulls it (k+1 readers on average), so the
@@ -80,53 +97,42 @@ __device__ __forceinline__ void join(Q4& x, const Q4& y)
 }
 
 // grid.x runs over (replica, panel, row group).  A thread owns one 32-byte column chunk of the
-// panel and walks kMergeIters rows of the block's row group.  Prologue: every row of the group
-// resolves its sources once (partner rows that answered, -1 otherwise) into shared memory, so
-// the streaming part has no dependent metadata loads.
+// panel and walks kMergeIters rows of the block's row group.  The sources of a row (the partners
+// that answered; an offline row has none and is copied) were resolved by k_gossip_resolve, so a
+// thread fetches them with one 16-byte load per row, all issued before the streaming part: no
+// shared memory, no barrier, no dependent metadata loads.
 // PUSH: full pairwise exchange, a row also takes the old rows of the nodes that pulled it
 // (their ids come from the per-round reverse lists).
 template <bool PUSH>
 __global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
                                                                      uint32_t n_panels, uint32_t groups_per_panel)
 {
-    __shared__ int4 s_src[kMergeThreads / 8 * kMergeIters];
-    __shared__ uint2 s_in[PUSH ? kMergeThreads / 8 * kMergeIters : 1];   // (offset, count) of the row's pullers
     const uint32_t b = blockIdx.x;
     const uint32_t per_replica = n_panels * groups_per_panel;
     const uint32_t r = b / per_replica;
     const uint32_t rem = b - r * per_replica;
     const uint32_t panel = rem / groups_per_panel, group = rem - panel * groups_per_panel;
     const uint32_t rstep = kMergeThreads >> chunk_shift;                  // rows covered by one pass of the block
-    const uint32_t rows_per_block = rstep * kMergeIters;
-    const uint32_t row0 = group * rows_per_block;
+    const uint32_t row0 = group * rstep * kMergeIters + (threadIdx.x >> chunk_shift);
     const size_t rbase = size_t(r) * n.N;
-    if (threadIdx.x < rows_per_block) {
-        int4 src = make_int4(-1, -1, -1, -1);
-        const uint32_t row = row0 + threadIdx.x;
-        if (row < n.N && n.online[rbase + row]) {
-            const int4 p4 = *reinterpret_cast<const int4*>(n.partner + (rbase + row) * 4);
-            const uint8_t* on = n.online + rbase;
-            src.x = p4.x >= 0 && on[p4.x] ? p4.x : -1;
-            src.y = p4.y >= 0 && on[p4.y] ? p4.y : -1;
-            src.z = p4.z >= 0 && on[p4.z] ? p4.z : -1;
-            src.w = p4.w >= 0 && on[p4.w] ? p4.w : -1;
-        }
-        s_src[threadIdx.x] = src;
-        if (PUSH) s_in[threadIdx.x] = row < n.N && n.online[rbase + row] ? make_uint2(n.in_off[rbase + row], n.in_deg[rbase + row])
-                                                                          : make_uint2(0, 0);
-    }
-    __syncthreads();
     const uint32_t c = panel * panel_cols + 4u * (threadIdx.x & ((1u << chunk_shift) - 1u));
     if (c >= n.ld) return;
+    int4 srcs[kMergeIters];
+    uint2 ins[PUSH ? kMergeIters : 1];                                    // (offset, count) of the row's reverse list
+#pragma unroll
+    for (int it = 0; it < kMergeIters; ++it) {
+        const uint32_t row = row0 + it * rstep;
+        srcs[it] = row < n.N ? __ldg(reinterpret_cast<const int4*>(n.partner) + rbase + row) : make_int4(-1, -1, -1, -1);
+        if (PUSH) ins[it] = row < n.N ? make_uint2(n.in_off[rbase + row], n.in_deg[rbase + row]) : make_uint2(0, 0);
+    }
     const uint32_t ld8 = n.ld * 8u;
     const char* in = reinterpret_cast<const char*>(n.view + rbase * n.ld + c);
     char* out = reinterpret_cast<char*>(n.view_new + rbase * n.ld + c);
-    uint32_t lr = threadIdx.x >> chunk_shift;
 #pragma unroll
-    for (int it = 0; it < kMergeIters; ++it, lr += rstep) {
-        const uint32_t row = row0 + lr;
+    for (int it = 0; it < kMergeIters; ++it) {
+        const uint32_t row = row0 + it * rstep;
         if (row >= n.N) break;
-        const int4 src = s_src[lr];
+        const int4 src = srcs[it];
         Q4 acc = ld32(in + uint64_t(row) * ld8);
         Q4 v0, v1, v2, v3;
         if (src.x >= 0) v0 = ld32(in + uint64_t(uint32_t(src.x)) * ld8);
@@ -138,9 +144,8 @@ __global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Ne
         if (src.z >= 0) join(acc, v2);
         if (src.w >= 0) join(acc, v3);
         if (PUSH) {
-            const uint2 in_list = s_in[lr];
-            const int32_t* who = n.pullers + rbase * 4 + in_list.x;
-            for (uint32_t j = 0; j < in_list.y; ++j) join(acc, ld32(in + uint64_t(uint32_t(who[j])) * ld8));
+            const int32_t* who = n.pullers + rbase * 4 + ins[it].x;
+            for (uint32_t j = 0; j < ins[it].y; ++j) join(acc, ld32(in + uint64_t(uint32_t(who[j])) * ld8));
         }
         st32_stream(out + uint64_t(row) * ld8, acc);
     }
@@ -157,7 +162,7 @@ __global__ void k_gossip_indeg(Net n)
     const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
 #pragma unroll
     for (int s = 0; s < 4; ++s)
-        if (p[s] >= 0 && n.online[size_t(r) * n.N + p[s]]) atomicAdd(&n.in_deg[size_t(r) * n.N + p[s]], 1u);
+        if (p[s] >= 0) atomicAdd(&n.in_deg[size_t(r) * n.N + p[s]], 1u);
 }
 
 // Exclusive prefix sum of the in-degrees of one replica (one block per replica).
@@ -203,7 +208,6 @@ __global__ void k_gossip_fill(Net n)
     for (int s = 0; s < 4; ++s) {
         if (p[s] < 0) continue;
         const size_t px = size_t(r) * n.N + p[s];
-        if (!n.online[px]) continue;
         const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
         n.pullers[size_t(r) * n.N * 4 + n.in_off[px] + k] = int32_t(i);
     }
@@ -228,10 +232,11 @@ __global__ void k_gossip_fixup(Net n)
     uint32_t marks = 0;
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        if (p[s] < 0) continue;
-        const size_t px = size_t(r) * n.N + p[s];
-        if (!n.online[px]) { atomicMax(vn + x * n.ld + p[s], n.view[x * n.ld + p[s]] | kOffBit); ++marks; }
-        else atomicMax(vn + px * n.ld + i, self);
+        if (p[s] == -1) continue;
+        if (p[s] < -1) {                             // chosen but dead: the pull failed
+            const uint32_t dead = uint32_t(-2 - p[s]);
+            atomicMax(vn + x * n.ld + dead, n.view[x * n.ld + dead] | kOffBit); ++marks;
+        } else atomicMax(vn + (size_t(r) * n.N + p[s]) * n.ld + i, self);
     }
     if (marks) atomicAdd(&n.stats[size_t(r) * sCount + sOfflineMarks], (unsigned long long)marks);
 }
@@ -262,6 +267,7 @@ void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c)
 {
     const dim3 pg((n.N + 127) / 128, n.Rp);
     { Timed t(c, kGossipPeer); k_gossip_peer<<<pg, 128, 0, c.stream>>>(n, round); }
+    { Timed t(c, kGossipPeer); k_gossip_resolve<<<pg, 128, 0, c.stream>>>(n); }
     const uint32_t pc = panel_columns(n);
     uint32_t shift = 0;
     while ((4u << shift) < pc) ++shift;                                   // 32-byte chunks per row segment = pc / 4
