@@ -30,7 +30,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return SO
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"] + os.environ.get("WWWS_NVCC_EXTRA", "").split()
+    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"] + __import__("shlex").split(os.environ.get("WWWS_NVCC_EXTRA", ""))
     cmd = [nvcc] + flags + (["-Xptxas", "-v"] if verbose else []) + ["-o", SO] + sources()
     subprocess.check_call(cmd)
     return SO

@@ -212,17 +212,7 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
         settle_one(n, r, uint32_t(first + idx), idx, n.origin[x], n.len_in[x], n.len_out[x], n.exec_a[x], n.exec_b[x], jd, n.outcome[x],
                    (n.rflags[x] & 1) != 0, s);
     }
-#pragma unroll
-    for (int k = 0; k < int(sSumLat); ++k) {
-        const uint32_t v = __reduce_add_sync(kFull, s.c[k]);
-        if ((threadIdx.x & 31) == 0) stats_add(bs, k, v);
-    }
-    unsigned long long sl = s.sum_lat;
-    for (int o = 16; o; o >>= 1) sl += __shfl_down_sync(kFull, sl, o);
-    if ((threadIdx.x & 31) == 0) stats_add(bs, sSumLat, sl);
-    unsigned long long dg = s.digest;
-    for (int o = 16; o; o >>= 1) dg += __shfl_down_sync(kFull, dg, o);
-    if ((threadIdx.x & 31) == 0) stats_add(bs, sPendingDigest, dg);
+    acc_flush_warp(bs, s);
     stats_end(n, bs, r);
 }
 

@@ -5,9 +5,10 @@
 // batch started.
 //
 // A thread scores its request's 32 candidates serially (the window is 256 contiguous bytes of
-// the origin's view row: eight 32-byte loads) and keeps the integer weights in shared memory,
-// laid out [candidate][slot] so that lanes never conflict and so that ANY thread of the block
-// can continue a request.  That is used for the duels: only a few requests per block become
+// the origin's view row: eight 32-byte loads) and keeps the fp32 scores in shared memory (the
+// integer weight is a function of the score alone and is recomputed where it is read: 4 bytes per
+// candidate instead of 8), laid out [candidate][slot] so that lanes never conflict and so that ANY
+// thread of the block can continue a request.  That is used for the duels: only a few requests per block become
 // duels, so instead of letting every warp run the long duel code for one or two of its lanes,
 // duel requests are queued in shared memory and picked up densely by the first threads of the
 // block after a barrier.
@@ -15,13 +16,28 @@
 
 namespace wwws {
 
+// Resident 128-thread blocks per SM the register budget is set for: at 7 (72 registers, 16 bytes
+// spilled) a 128,000-request launch is a single wave on 148 SMs; shared memory (18 KiB per block)
+// would allow 12.
+constexpr int kStepBlocksPerSM = 7;
+// Unroll factor of the scoring loop over the four 8-candidate groups: 2 keeps two window loads in
+// flight per thread at half the code of a full unroll.
+constexpr int kScoreUnroll = 2;
+
 template <int BT> struct StepShared {
-    unsigned long long W[kWin][BT];      // integer weights, 0 = not in play
+    float S[kWin][BT];                   // fp32 scores of the candidates still in play, 0 = not in play
     BlockStats stats;
     uint32_t n_duel;
     uint16_t queue[BT];                  // slots whose request became a duel
     struct Ctx { int32_t a; uint32_t blk; uint32_t draws_probes_near; } ctx[BT];
 };
+
+// The integer weight that candidate_weight() derives from a score.
+__device__ __forceinline__ uint64_t weight_of(float sc)
+{
+    const float scaled = __fmul_rn(sc, 256.0f);
+    return scaled >= 72057594037927936.0f ? (1ull << 56) : __float2ull_rz(scaled);
+}
 
 // Draw state of one request, held by the thread that is working on it.
 struct Draws {
@@ -45,12 +61,12 @@ __device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, 
         int pick = -1;
 #pragma unroll 8
         for (int c = 0; c < int(kWin); ++c) {
-            const uint64_t w = sh.W[c][slot];
+            const uint64_t w = weight_of(sh.S[c][slot]);
             if (w > m) { m2 = m; m = w; pick = c; }
             else if (w > m2) m2 = w;
         }
         if (m2 != 0 && m - m2 <= m / 100000ull) d.near = true;
-        sh.W[pick][slot] = 0;
+        sh.S[pick][slot] = 0.0f;
         const int g = pick >> 3;
         if (g == 0) d.G0 -= m; else if (g == 1) d.G1 -= m; else if (g == 2) d.G2 -= m; else d.G3 -= m;
         return pick;
@@ -67,7 +83,7 @@ __device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, 
     uint64_t wp = 0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const uint64_t w = sh.W[8 * g + j][slot];
+        const uint64_t w = weight_of(sh.S[8 * g + j][slot]);
         if (pick < 0) {
             if (r64 < lo + w) { pick = 8 * g + j; wp = w; }
             else lo += w;
@@ -75,7 +91,7 @@ __device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, 
     }
     const uint64_t m1 = r64 - lo, m2 = lo + wp - 1 - r64;
     if ((m1 < m2 ? m1 : m2) <= S / 100000ull) d.near = true;
-    sh.W[pick][slot] = 0;
+    sh.S[pick][slot] = 0.0f;
     if (g == 0) d.G0 -= wp; else if (g == 1) d.G1 -= wp; else if (g == 2) d.G2 -= wp; else d.G3 -= wp;
     return pick;
 }
@@ -94,19 +110,6 @@ __device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg
     return on && cap != 0 && !util_at_least(cap, queued, n.util_window_ms, accept_util) && u < accept_freq;
 }
 
-template <int BT>
-__device__ __forceinline__ int find_peer(const Net& n, StepShared<BT>& sh, uint32_t slot, Draws& d, uint32_t r, uint32_t rg,
-                                         uint32_t q, uint32_t blk)
-{
-    while (d.n_probes < n.max_probes) {
-        const int pick = draw_candidate(n, sh, slot, d, q, rg);
-        if (pick < 0) break;
-        d.n_probes++;
-        if (probe_peer(n, r, rg, q, blk, pick)) return int(kWin * blk + pick);
-    }
-    return -1;
-}
-
 // Scores the window of request (o, blk) into shared memory; returns the four group sums through d
 // and the lane-ascending fp32 sum of the scores.
 template <int BT>
@@ -116,7 +119,7 @@ __device__ __forceinline__ float score_window(const Net& n, StepShared<BT>& sh, 
     const uint64_t* win = n.view + (size_t(r) * n.N + o) * n.ld + kWin * blk;
     const float* wled = n.w_led + size_t(r) * n.N;
     float ssum = 0.0f;
-#pragma unroll
+#pragma unroll kScoreUnroll
     for (int g = 0; g < 4; ++g) {
         uint64_t gsum = 0;
 #pragma unroll
@@ -129,10 +132,10 @@ __device__ __forceinline__ float score_window(const Net& n, StepShared<BT>& sh, 
                 const uint32_t id = kWin * blk + c0 + j;
                 const float wl = id < n.N ? wled[id] : 0.0f;
                 float sc;
-                uint64_t W = candidate_weight(n, o, id, e[j], wl, sc);
-                if (!(keep >> (c0 + j) & 1u)) W = 0;                                       // lanes already drawn (duel pass)
-                sh.W[c0 + j][slot] = W;
-                gsum += W;
+                const uint64_t W = candidate_weight(n, o, id, e[j], wl, sc);              // sc = 0 when W = 0
+                const bool in_play = keep >> (c0 + j) & 1u;                                // not drawn already (duel pass)
+                sh.S[c0 + j][slot] = in_play ? sc : 0.0f;
+                gsum += in_play ? W : 0ull;
                 ssum = __fadd_rn(ssum, sc);                                                // lane-ascending fp32 sum
             }
         }
@@ -144,132 +147,137 @@ __device__ __forceinline__ float score_window(const Net& n, StepShared<BT>& sh, 
 // What a launch does: the whole step, or one of the two calls it replaces on large batches.
 enum : int { kModeFused = 0, kModeDispatch = 1, kModeDuel = 2 };
 
+// The kernel makes two passes over the same code.  Pass 0: every thread takes its own request
+// (origin decision, scoring, search for the executor).  Pass 1, after a barrier: the first
+// threads of the block take the requests that became duels (search for the challenger, then the
+// judges).  Both passes share one draw/probe loop, one result writer and one settlement, so the
+// machine code holds each of those long sequences once: the kernel is bound by instruction
+// fetch when many blocks at different points of a large program share an SM.
 template <int BT, int MODE>
-__global__ void __launch_bounds__(BT, BT == 128 ? 5 : 1) k_step_fused(Net n, uint64_t first, uint32_t count)
+__global__ void __launch_bounds__(BT, BT == 128 ? kStepBlocksPerSM : 1) k_step_fused(Net n, uint64_t first, uint32_t count)
 {
     __shared__ StepShared<BT> sh;
     stats_begin(sh.stats);                       // barrier inside
     if (threadIdx.x == 0) sh.n_duel = 0;
     __syncthreads();
     const uint32_t r = blockIdx.y, rg = r + n.replica_offset;
-    const uint32_t slot = threadIdx.x;
-    const uint32_t idx = blockIdx.x * BT + slot;
+    const size_t pbase = size_t(r) * n.N;
     SettleAcc acc; acc_zero(acc);
 
-    if (MODE != kModeDuel) {
-        // ---- dispatch (D1..D6), one request per thread -------------------------------------
-        if (idx < count) {
-            const uint32_t q = uint32_t(first + idx);
-            const size_t x = size_t(r) * n.Q + first + idx;
-            const uint32_t o = n.origin[x];
-            const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
-            int a;
-            float sa = 0.0f, ssum = 0.0f;
-            Draws d;
-            d.G0 = d.G1 = d.G2 = d.G3 = 0; d.n_draws = 0; d.n_probes = 0; d.near = false; d.y_slot = 0xffffffffu;
-            uint32_t blk = 0;
-            bool duel = false, scored = false;
-            if (origin_offloads(n, r, o, rx, a)) {
-                const int local_code = a;
-                blk = pick_block(n, o, rx.w[2]);
-                ssum = score_window<BT>(n, sh, slot, r, o, blk, 0xffffffffu, d);
-                scored = true;
-                a = find_peer<BT>(n, sh, slot, d, r, rg, q, blk);
-                if (a >= 0) {
-                    if (n.score_a) {
-                        float sc;
-                        candidate_weight(n, o, uint32_t(a), n.view[(size_t(r) * n.N + o) * n.ld + a], n.w_led[size_t(r) * n.N + a], sc);
-                        sa = sc;
-                    }
-                    duel = ppm(rx.w[1]) < n.p_duel;
-                } else a = local_code == -4 ? -4 : -2;
-            }
-            n.exec_a[x] = a;
-            if (n.score_a) n.score_a[x] = sa;
-            if (n.score_sum) n.score_sum[x] = ssum;
-            if (MODE == kModeFused && duel) {
-                const uint32_t k = atomicAdd(&sh.n_duel, 1u);
-                sh.queue[k] = uint16_t(slot);
-                sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
-                sh.ctx[slot].draws_probes_near = d.n_draws | (d.n_probes << 8) | (d.near ? 1u << 16 : 0u);
-            } else {
-                n.exec_b[x] = -1; n.outcome[x] = 0; n.rflags[x] = d.near ? 1 : 0;
-                *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(-1, -1, -1, -1);
-                acc.c[sProbes] += d.n_probes;
-                if (MODE == kModeFused) {
-                    const int jd[4] = { -1, -1, -1, -1 };
-                    settle_one(n, r, q, idx, o, n.len_in[x], n.len_out[x], a, -1, jd, 0, d.near, acc);
-                } else {
-                    // continuation for the duel call: lanes still in play, draws and probes used
-                    uint32_t mask = 0;
-                    if (scored) {
-#pragma unroll
-                        for (int c = 0; c < int(kWin); ++c) mask |= (sh.W[c][slot] != 0 ? 1u : 0u) << c;
-                    }
-                    n.cont[size_t(r) * n.max_batch + idx] = make_uint2(mask, d.n_draws | (d.n_probes << 8));
-                }
-            }
-        }
-    } else {
-        // ---- duel call: requests flagged as duels re-create their window and queue up ----------
-        if (idx < count) {
-            const uint32_t q = uint32_t(first + idx);
-            const size_t x = size_t(r) * n.Q + first + idx;
-            const int a = n.exec_a[x];
-            if (a >= 0) {
-                const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
-                if (ppm(rx.w[1]) < n.p_duel) {
-                    const uint32_t o = n.origin[x];
-                    const uint2 ct = n.cont[size_t(r) * n.max_batch + idx];
-                    const uint32_t blk = pick_block(n, o, rx.w[2]);
-                    Draws d;
-                    score_window<BT>(n, sh, slot, r, o, blk, ct.x, d);
-                    const uint32_t k = atomicAdd(&sh.n_duel, 1u);
-                    sh.queue[k] = uint16_t(slot);
-                    sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
-                    sh.ctx[slot].draws_probes_near = (ct.y & 0xffffu) | ((n.rflags[x] & 1u) << 16);
-                }
-            }
-        }
-    }
-    __syncthreads();
-
-    // ---- duel-and-judge (J2, J3) for the queued requests, densely -----------------------------
-    if (MODE != kModeDispatch && threadIdx.x < sh.n_duel) {
-        const uint32_t ds = sh.queue[threadIdx.x];
-        const uint32_t didx = blockIdx.x * BT + ds;
-        const uint32_t q = uint32_t(first + didx);
-        const size_t x = size_t(r) * n.Q + first + didx;
-        const int a = sh.ctx[ds].a;
-        const uint32_t blk = sh.ctx[ds].blk, packed = sh.ctx[ds].draws_probes_near;
+#pragma unroll 1
+    for (int pass = 0; pass < (MODE == kModeDispatch ? 1 : 2); ++pass) {
+        uint32_t slot = threadIdx.x;             // the request of the block this thread works on
+        bool search = false, finish = false, duel_if_found = false, scored = false;
+        int a = -1, local_code = -1;
+        uint32_t blk = 0, o = 0, probes0 = 0;
+        float ssum = 0.0f;
         Draws d;
-        d.n_draws = packed & 0xffu; d.n_probes = (packed >> 8) & 0xffu; d.near = (packed >> 16) & 1u; d.y_slot = 0xffffffffu;
-        const uint32_t probes0 = d.n_probes;
-        uint64_t gs[4];
+        d.G0 = d.G1 = d.G2 = d.G3 = 0; d.n_draws = 0; d.n_probes = 0; d.near = false; d.y_slot = 0xffffffffu;
+
+        if (pass == 0) {
+            const uint32_t idx = blockIdx.x * BT + slot;
+            if (idx < count) {
+                const uint32_t q = uint32_t(first + idx);
+                const size_t x = size_t(r) * n.Q + first + idx;
+                const Rnd4 rx = draw(n, q, 0, rg, kOrigin);
+                if (MODE != kModeDuel) {
+                    // ---- dispatch (D1..D4): origin decision and scoring ---------------------
+                    o = n.origin[x];
+                    finish = true;
+                    if (origin_offloads(n, r, o, rx, a)) {
+                        local_code = a;
+                        blk = pick_block(n, o, rx.w[2]);
+                        ssum = score_window<BT>(n, sh, slot, r, o, blk, 0xffffffffu, d);
+                        scored = search = true;
+                        duel_if_found = ppm(rx.w[1]) < n.p_duel;
+                    }
+                } else {
+                    // ---- duel call: requests flagged as duels re-create their window and queue up
+                    const int a0 = n.exec_a[x];
+                    if (a0 >= 0 && ppm(rx.w[1]) < n.p_duel) {
+                        const uint2 ct = n.cont[size_t(r) * n.max_batch + idx];
+                        blk = pick_block(n, n.origin[x], rx.w[2]);
+                        score_window<BT>(n, sh, slot, r, n.origin[x], blk, ct.x, d);
+                        const uint32_t k = atomicAdd(&sh.n_duel, 1u);
+                        sh.queue[k] = uint16_t(slot);
+                        sh.ctx[slot].a = a0; sh.ctx[slot].blk = blk;
+                        sh.ctx[slot].draws_probes_near = (ct.y & 0xffffu) | ((n.rflags[x] & 1u) << 16);
+                    }
+                }
+            }
+        } else {
+            // ---- duel-and-judge (J2, J3) for the queued requests, densely ----------------------
+            __syncthreads();
+            if (threadIdx.x < sh.n_duel) {
+                slot = sh.queue[threadIdx.x];
+                a = sh.ctx[slot].a; blk = sh.ctx[slot].blk;
+                const uint32_t packed = sh.ctx[slot].draws_probes_near;
+                d.n_draws = packed & 0xffu; d.n_probes = (packed >> 8) & 0xffu; d.near = (packed >> 16) & 1u;
+                probes0 = MODE == kModeDuel ? d.n_probes : 0u;
+                uint64_t gs[4];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            gs[g] = 0;
+                for (int g = 0; g < 4; ++g) {
+                    gs[g] = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) gs[g] += sh.W[8 * g + j][ds];
+                    for (int j = 0; j < 8; ++j) gs[g] += weight_of(sh.S[8 * g + j][slot]);
+                }
+                d.G0 = gs[0]; d.G1 = gs[1]; d.G2 = gs[2]; d.G3 = gs[3];
+                search = finish = true;
+            }
         }
-        d.G0 = gs[0]; d.G1 = gs[1]; d.G2 = gs[2]; d.G3 = gs[3];
-        int b = find_peer<BT>(n, sh, ds, d, r, rg, q, blk);
+        const uint32_t idx = blockIdx.x * BT + slot;
+        const uint32_t q = uint32_t(first + idx);
+        const size_t x = size_t(r) * n.Q + first + idx;
+
+        // ---- D5, D6 / J2: draw and probe until a peer accepts; in pass 1 go on drawing judges ------
+        int found = -1, nj = 0;
         int jd[4] = { -1, -1, -1, -1 };
-        uint32_t oc = 4;
-        if (b >= 0) {
-            int nj = 0;
-            while (nj < int(n.n_judges)) {
-                const int pick = draw_candidate(n, sh, ds, d, q, rg);
+        if (search) {
+            for (;;) {
+                if (found < 0) { if (d.n_probes >= n.max_probes) break; }
+                else if (pass == 0 || nj >= int(n.n_judges)) break;
+                const int pick = draw_candidate(n, sh, slot, d, q, rg);
                 if (pick < 0) break;
                 const int id = int(kWin * blk + pick);
-                if (n.online[size_t(r) * n.N + id]) {
+                if (found < 0) {
+                    d.n_probes++;
+                    if (probe_peer(n, r, rg, q, blk, pick)) found = id;
+                } else if (n.online[pbase + id]) {
                     if (nj == 0) jd[0] = id; else if (nj == 1) jd[1] = id; else if (nj == 2) jd[2] = id; else jd[3] = id;
                     ++nj;
                 }
             }
-            if (nj == 0) b = -1;
-            else {
-                const uint64_t thr = ((1ull << 32) + n.quality[size_t(r) * n.N + a] - n.quality[size_t(r) * n.N + b]) >> 1;
+        }
+
+        int b = -1;
+        uint32_t oc = 0;
+        if (pass == 0) {
+            if (MODE != kModeDuel && finish) {
+                bool duel = false;
+                float sa = 0.0f;
+                if (search) {
+                    if (found >= 0) {
+                        a = found;
+                        duel = duel_if_found;
+                        if (n.score_a) candidate_weight(n, o, uint32_t(a), n.view[(pbase + o) * n.ld + a], n.w_led[pbase + a], sa);
+                    } else a = local_code == -4 ? -4 : -2;
+                }
+                n.exec_a[x] = a;
+                if (n.score_a) n.score_a[x] = sa;
+                if (n.score_sum) n.score_sum[x] = ssum;
+                if (MODE == kModeFused && duel) {
+                    const uint32_t k = atomicAdd(&sh.n_duel, 1u);
+                    sh.queue[k] = uint16_t(slot);
+                    sh.ctx[slot].a = a; sh.ctx[slot].blk = blk;
+                    sh.ctx[slot].draws_probes_near = d.n_draws | (d.n_probes << 8) | (d.near ? 1u << 16 : 0u);
+                    finish = false;                      // settled in pass 1
+                }
+            }
+        } else if (finish) {
+            oc = 4;
+            if (found >= 0 && nj > 0) {
+                b = found;
+                const uint64_t thr = ((1ull << 32) + n.quality[pbase + a] - n.quality[pbase + b]) >> 1;
                 int votes_a = 0;
                 for (int l = 0; l < nj; ++l) {
                     const Rnd4 y = draw(n, q, uint32_t(l), rg, kJudge);
@@ -278,31 +286,30 @@ __global__ void __launch_bounds__(BT, BT == 128 ? 5 : 1) k_step_fused(Net n, uin
                     votes_a += va;
                 }
                 oc = 2 * votes_a > nj ? 1u : (2 * votes_a < nj ? 2u : 3u);
-            }
+            } else jd[0] = jd[1] = jd[2] = jd[3] = -1;
+            o = n.origin[x];
         }
-        if (oc == 4) { b = -1; jd[0] = jd[1] = jd[2] = jd[3] = -1; }
-        n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = d.near ? 1 : 0;
-        *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
-        if (MODE == kModeFused) {
-            acc.c[sProbes] += d.n_probes;
-            settle_one(n, r, q, didx, n.origin[x], n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
-        } else {
-            acc.c[sProbes] += d.n_probes - probes0;
+
+        // ---- results and settlement (S1..S4) of the request this pass completed -----------------
+        if (finish) {
+            n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = d.near ? 1 : 0;
+            *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
+            acc.probes += d.n_probes - probes0;
+            if (MODE == kModeFused) settle_one(n, r, q, idx, o, n.len_in[x], n.len_out[x], a, b, jd, oc, d.near, acc);
+            if (MODE == kModeDispatch) {
+                // continuation for the duel call: lanes still in play, draws and probes used
+                uint32_t mask = 0;
+                if (scored) {
+#pragma unroll
+                    for (int c = 0; c < int(kWin); ++c) mask |= (sh.S[c][slot] != 0.0f ? 1u : 0u) << c;
+                }
+                n.cont[size_t(r) * n.max_batch + idx] = make_uint2(mask, d.n_draws | (d.n_probes << 8));
+            }
         }
     }
 
     // ---- counters: warp reduce, block reduce, one atomic per counter and block ---------------
-#pragma unroll
-    for (int k = 0; k < int(sSumLat); ++k) {
-        const uint32_t v = __reduce_add_sync(kFull, acc.c[k]);
-        if ((threadIdx.x & 31) == 0) stats_add(sh.stats, k, v);
-    }
-    unsigned long long sl = acc.sum_lat;
-    for (int o = 16; o; o >>= 1) sl += __shfl_down_sync(kFull, sl, o);
-    if ((threadIdx.x & 31) == 0) stats_add(sh.stats, sSumLat, sl);
-    unsigned long long dg = acc.digest;
-    for (int o = 16; o; o >>= 1) dg += __shfl_down_sync(kFull, dg, o);
-    if ((threadIdx.x & 31) == 0) stats_add(sh.stats, sPendingDigest, dg);
+    acc_flush_warp(sh.stats, acc);
     stats_end(n, sh.stats, r);
 }
 

@@ -89,19 +89,30 @@ __device__ __forceinline__ bool origin_offloads(const Net& n, uint32_t r, uint32
 
 // 64-bit by 32-bit unsigned division; the common case (numerator below 2^32) takes the short
 // 32-bit path instead of the long emulated 64-bit one.
+static __device__ __noinline__ uint64_t udiv64_long(uint64_t t, uint32_t d) { return t / d; }   // one copy of the long path
 __device__ __forceinline__ uint64_t udiv64by32(uint64_t t, uint32_t d)
 {
-    return (t >> 32) == 0 ? uint64_t(uint32_t(t) / d) : t / d;
+    return (t >> 32) == 0 ? uint64_t(uint32_t(t) / d) : udiv64_long(t, d);
 }
 
 // ---- settlement of one request (one thread) ----------------------------------------------------
 
 __device__ __forceinline__ void add64(long long* p, long long v) { atomicAdd((unsigned long long*)p, (unsigned long long)v); }
 
+// Counters of the (at most two) requests a thread settles.  The twelve event counters other than
+// the probe count stay below 8 per thread, so they are kept as 8-bit fields, four to a word, and
+// a warp's sum of a field (at most 32 * 7) still fits its field: three reductions instead of twelve.
 struct SettleAcc {
-    uint32_t c[sSumLat];           // counters before sSumLat are small
+    uint32_t p[3];                 // field f of counter k: f = k below sProbes, k - 1 above
+    uint32_t probes;
     unsigned long long sum_lat;
     unsigned long long digest;     // wrapping sum of the record hashes of this thread's requests
+    __device__ __forceinline__ void add(uint32_t k, uint32_t v = 1u)
+    {
+        if (k == sProbes) { probes += v; return; }
+        const uint32_t f = k < sProbes ? k : k - 1;
+        p[f >> 2] += v << (8u * (f & 3u));
+    }
 };
 
 // With exact intra-batch queueing (flag 16) the latency of a request depends on the work that
@@ -129,18 +140,18 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
     }
     const size_t base = size_t(r) * n.N;
     const uint64_t work = uint64_t(li) + lo;
-    s.c[sRequests]++;
-    if (near) s.c[sNear]++;
-    if (a == -3) { s.c[sDropped]++; return; }
-    if (a == -4) { s.c[sFailed]++; return; }
+    s.add(sRequests);
+    if (near) s.add(sNear);
+    if (a == -3) { s.add(sDropped); return; }
+    if (a == -4) { s.add(sFailed); return; }
     uint32_t ex;
     if (a < 0) {
-        s.c[a == -1 ? sLocal : sFallback]++;
+        if (a == -1) s.add(sLocal); else s.add(sFallback);
         add64(&n.d_backlog[base + o], (long long)work);
         atomicAdd(&n.served_local[base + o], 1ull);
         ex = o;
     } else {
-        s.c[sDelegated]++;
+        s.add(sDelegated);
         const uint64_t key = chain_key(n, r);
         long long pay = n.R;
         s.digest += record_hash(key, q, opPay, o, -n.R) + record_hash(key, q, opEarn, uint32_t(a), n.R);
@@ -148,8 +159,8 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
         add64(&n.d_backlog[base + a], (long long)work);
         atomicAdd(&n.served[base + a], 1ull);
         ex = uint32_t(a);
-        if (oc != 0) s.c[sDuel]++;
-        if (oc == 4) s.c[sDuelCancelled]++;
+        if (oc != 0) s.add(sDuel);
+        if (oc == 4) s.add(sDuelCancelled);
         if (oc >= 1 && oc <= 3) {
             pay += n.R;
             s.digest += record_hash(key, q, opPayChallenger, o, -n.R) + record_hash(key, q, opEarnChallenger, uint32_t(b), n.R);
@@ -162,8 +173,8 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
 #pragma unroll
             for (int l = 0; l < 4; ++l)
                 if (jd[l] >= 0) { add64(&n.d_backlog[base + jd[l]], (long long)(uint64_t(li) + 2ull * lo)); ++nj; }
-            s.c[sJudgeEvals] += nj;
-            if (oc == 3) s.c[sDraw]++;
+            s.add(sJudgeEvals, uint32_t(nj));
+            if (oc == 3) s.add(sDraw);
             else {
                 const int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
                 const long long pot = n.P - n.R_add, share = n.judge_share[nj - 1];
@@ -189,22 +200,32 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
     const uint64_t ideal = udiv64by32(work * 1000ull + n.cap_ref - 1, n.cap_ref);
     const uint64_t deadline = udiv64by32(uint64_t(n.slo_num) * ideal, n.slo_den);
     s.sum_lat += lat;
-    if (lat <= deadline) s.c[sSloMet]++;
+    if (lat <= deadline) s.add(sSloMet);
 }
 
 __device__ __forceinline__ void acc_zero(SettleAcc& s)
 {
-#pragma unroll
-    for (int k = 0; k < int(sSumLat); ++k) s.c[k] = 0;
+    s.p[0] = s.p[1] = s.p[2] = 0; s.probes = 0;
     s.sum_lat = 0;
     s.digest = 0;
 }
-__device__ __forceinline__ void acc_flush(BlockStats& bs, const SettleAcc& s)
+
+// Warp sums of a thread's counters, added to the block's counters by lane 0 (all lanes call).
+__device__ __forceinline__ void acc_flush_warp(BlockStats& bs, const SettleAcc& s)
 {
+    const uint32_t w0 = __reduce_add_sync(kFull, s.p[0]), w1 = __reduce_add_sync(kFull, s.p[1]), w2 = __reduce_add_sync(kFull, s.p[2]);
+    const uint32_t pr = __reduce_add_sync(kFull, s.probes);
+    unsigned long long sl = s.sum_lat, dg = s.digest;
 #pragma unroll
-    for (int k = 0; k < int(sSumLat); ++k) stats_add(bs, k, s.c[k]);
-    stats_add(bs, sSumLat, s.sum_lat);
-    stats_add(bs, sPendingDigest, s.digest);
+    for (int o = 16; o; o >>= 1) { sl += __shfl_down_sync(kFull, sl, o); dg += __shfl_down_sync(kFull, dg, o); }
+    if ((threadIdx.x & 31) == 0) {
+        const uint32_t w[3] = { w0, w1, w2 };
+#pragma unroll
+        for (uint32_t f = 0; f < 12; ++f) stats_add(bs, f < sProbes ? f : f + 1, (w[f >> 2] >> (8u * (f & 3u))) & 0xffu);
+        stats_add(bs, sProbes, pr);
+        stats_add(bs, sSumLat, sl);
+        stats_add(bs, sPendingDigest, dg);
+    }
 }
 
 }  // namespace wwws

@@ -136,7 +136,7 @@ __device__ __forceinline__ uint64_t chain_key(const Net& n, uint32_t r)
 }
 // Hash of one ledger record: request q moves `amount` credits on `peer`'s account, for reason `kind`.
 enum : uint32_t { opPay = 1, opEarn = 2, opPayChallenger = 3, opEarnChallenger = 4, opPenalty = 5, opReward = 6, opJudge = 7 };
-__device__ __forceinline__ uint64_t record_hash(uint64_t key, uint32_t q, uint32_t kind, uint32_t peer, int64_t amount)
+static __device__ __noinline__ uint64_t record_hash(uint64_t key, uint32_t q, uint32_t kind, uint32_t peer, int64_t amount)
 {
     return mix64(mix64(key ^ (uint64_t(q) << 32 | uint64_t(kind) << 24 | peer)) + uint64_t(amount));
 }
