@@ -34,7 +34,7 @@ DEFAULT_WORKLOAD = "adversarial16k"          # the largest single-GPU configurat
 # DRAM traffic (read + write) of one k_gossip_merge pass over one replica, from the ncu capture
 # summarised in profiles/k_gossip_merge_adversarial16k_1replica.md; a launch over Rp replicas is
 # Rp such passes back to back (replica-major grid), so traffic scales with the replica count.
-NCU_MERGE_TRAFFIC = {"n_peers": 16384, "fanout_k": 4, "flags": 3, "bytes_per_replica": 2.1932e9 + 2.1138e9}
+NCU_MERGE_TRAFFIC = {"n_peers": 16384, "fanout_k": 4, "flags": 3, "bytes_per_replica": 2.1897e9 + 2.1133e9}
 
 
 def measured_peaks():
