@@ -182,6 +182,29 @@ def test_push_pull_gossip_matches_oracle(n_peers, k, churn):
     assert_same_state(g, o, "push-pull end", upto=wl.n_requests)
 
 
+@pytest.mark.parametrize("n_peers,k,churn,stale", [(1024, 4, 60_000, 5), (1100, 4, 60_000, 0), (300, 2, 0, 3), (40, 1, 200_000, 0),
+                                                   (2100, 3, 30_000, 2)])
+def test_gossip_rounds_on_uniform_and_ragged_rows_match_oracle(n_peers, k, churn, stale):
+    """Several gossip rounds per step on row lengths that are and are not a multiple of the
+    panel width (1100 peers pad to 1120 columns, 2100 to 2112), with churn and stale initial views."""
+    wl = synth.make_workload("churn4k", n_replicas=3, n_requests=4000, n_peers=n_peers)
+    wl.settings.fanout_k = k
+    wl.settings.p_leave_ppm = wl.settings.p_join_ppm = churn
+    wl.settings.init_stale_max = stale
+    g, o = _pair(wl)
+    for s in range(4):
+        g.advance_time(wl.step_now_ms(s)); o.advance_time(wl.step_now_ms(s))
+        for _ in range(3):
+            g.gossip_round(); o.gossip_round()
+        assert_same_state(g, o, f"gossip x3, step {s}")
+        first = s * wl.batch
+        g.dispatch_batch(first, wl.batch); o.dispatch_batch(first, wl.batch)
+        g.duel_judge(); o.duel_judge()
+        g.settle_credits(True); o.settle_credits(True)
+    assert_same_state(g, o, "gossip x3, end", upto=4 * wl.batch)
+    assert g.stats_dict()["rounds"] == 3 * 12
+
+
 @pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiers64", dict(n_requests=5000)),
                                      ("zipf1k", dict(n_replicas=3, n_requests=2500, n_peers=200))])
 def test_fifo_queueing_matches_oracle(name, kw):
