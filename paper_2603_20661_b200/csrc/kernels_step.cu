@@ -32,13 +32,6 @@ template <int BT> struct StepShared {
     struct Ctx { int32_t a; uint32_t blk; uint32_t draws_probes_near; } ctx[BT];
 };
 
-// The integer weight that candidate_weight() derives from a score.
-__device__ __forceinline__ uint64_t weight_of(float sc)
-{
-    const float scaled = __fmul_rn(sc, 256.0f);
-    return scaled >= 72057594037927936.0f ? (1ull << 56) : __float2ull_rz(scaled);
-}
-
 // Draw state of one request, held by the thread that is working on it.
 struct Draws {
     uint64_t G0, G1, G2, G3;             // sums of the four 8-candidate groups still in play
@@ -94,20 +87,6 @@ __device__ __forceinline__ int draw_candidate(const Net& n, StepShared<BT>& sh, 
     sh.S[pick][slot] = 0.0f;
     if (g == 0) d.G0 -= wp; else if (g == 1) d.G1 -= wp; else if (g == 2) d.G2 -= wp; else d.G3 -= wp;
     return pick;
-}
-
-// D6: the drawn candidate answers by its true state and its own accept policy.  All five values
-// are loaded at once and the probe's random word is computed while they are in flight: one
-// memory round trip per probe instead of a chain of dependent ones.
-__device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg, uint32_t q, uint32_t blk, int pick)
-{
-    const size_t x = size_t(r) * n.N + kWin * blk + pick;
-    const uint32_t cap = n.cap_eff[x];
-    const uint8_t on = n.online[x];
-    const int64_t queued = n.backlog[x];
-    const uint32_t accept_util = n.accept_util_pm[x], accept_freq = n.accept_ppm[x];
-    const uint32_t u = ppm(draw(n, q, uint32_t(pick) >> 2, rg, kProbe).w[pick & 3]);
-    return on && cap != 0 && !util_at_least(cap, queued, n.util_window_ms, accept_util) && u < accept_freq;
 }
 
 // Scores the window of request (o, blk) into shared memory; returns the four group sums through d
@@ -325,6 +304,8 @@ static void launch_by_size(const Net& n, uint64_t first, uint32_t count, const L
 
 void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
+    // launches that leave most of the GPU empty share a request among several lanes
+    if (const int lanes = step_lanes_for(uint64_t(count) * n.Rp)) { launch_step_lanes(n, first, count, lanes, c); return; }
     Timed t(c, kStepFused);
     launch_by_size<kModeFused>(n, first, count, c);
 }

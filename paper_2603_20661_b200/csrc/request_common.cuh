@@ -71,6 +71,27 @@ __device__ __forceinline__ uint64_t candidate_weight(const Net& n, uint32_t o, u
     return W;
 }
 
+// The integer weight that candidate_weight() derives from a score.
+__device__ __forceinline__ uint64_t weight_of(float sc)
+{
+    const float scaled = __fmul_rn(sc, 256.0f);
+    return scaled >= 72057594037927936.0f ? (1ull << 56) : __float2ull_rz(scaled);
+}
+
+// D6: the drawn candidate answers by its true state and its own accept policy.  All five values
+// are loaded at once and the probe's random word is computed while they are in flight: one
+// memory round trip per probe instead of a chain of dependent ones.
+__device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg, uint32_t q, uint32_t blk, int pick)
+{
+    const size_t x = size_t(r) * n.N + kWin * blk + pick;
+    const uint32_t cap = n.cap_eff[x];
+    const uint8_t on = n.online[x];
+    const int64_t queued = n.backlog[x];
+    const uint32_t accept_util = n.accept_util_pm[x], accept_freq = n.accept_ppm[x];
+    const uint32_t u = ppm(draw(n, q, uint32_t(pick) >> 2, rg, kProbe).w[pick & 3]);
+    return on && cap != 0 && !util_at_least(cap, queued, n.util_window_ms, accept_util) && u < accept_freq;
+}
+
 // Origin side of dispatch (D1, D2).  Returns 1 if the request goes to the network, else
 // writes the local / dropped / failed code to `code`.
 __device__ __forceinline__ bool origin_offloads(const Net& n, uint32_t r, uint32_t o, const Rnd4& rx, int& code)

@@ -50,6 +50,8 @@ void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchC
 void launch_duel(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_settle(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
+int step_lanes_for(uint64_t total_requests);
+void launch_step_lanes(const Net& n, uint64_t first, uint32_t count, int lanes, const LaunchCtx& c);
 void launch_dispatch_threads(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_duel_threads(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 
