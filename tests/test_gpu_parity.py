@@ -108,6 +108,24 @@ def test_fused_step_matches_oracle(name, kw, steps):
     assert_same_state(g, o, "fused end", upto=wl.n_requests)
 
 
+@pytest.mark.parametrize("batch,flags", [(250, 3), (1500, 3), (5000, 3), (10000, 3), (250, 7), (1500, 7), (1500, 19)],
+                         ids=["8_lanes", "4_lanes", "thread_blocks_of_32", "thread_blocks_of_128", "8_lanes_greedy", "4_lanes_greedy",
+                              "4_lanes_fifo"])
+def test_fused_step_at_every_launch_size_matches_oracle(batch, flags):
+    """The fused step picks its kernel by launch size (8 or 4 lanes per request, one thread per
+    request in blocks of 32 or 128): 8 replicas x batch = 2,000 / 12,000 / 40,000 / 80,000 requests."""
+    wl = synth.make_workload("zipf1k", n_replicas=8, n_requests=2 * batch, n_peers=300)
+    wl.batch = batch
+    wl.settings.flags = flags
+    wl.settings.p_duel_ppm = 150_000
+    g, o = _pair(wl)
+    for s in range(2):
+        g.step(s * batch, batch, wl.step_now_ms(s), s == 0, s == 1)
+        o.run_step(s * batch, batch, wl.step_now_ms(s), s == 0, s == 1)
+        assert_same_state(g, o, f"batch {batch} step {s}", upto=(s + 1) * batch, views=s == 0)
+    assert o.stats_dict()["n_duel"] > 0.05 * o.stats_dict()["n_delegated"] > 0
+
+
 def test_step_host_roundtrip_matches_oracle():
     import torch
     from paper_2603_20661_b200.binding import Network
