@@ -16,8 +16,8 @@
 
 namespace wwws {
 
-// Resident 128-thread blocks per SM the register budget is set for: at 7 (72 registers, 16 bytes
-// spilled) a 128,000-request launch is a single wave on 148 SMs; shared memory (18 KiB per block)
+// Resident 128-thread blocks per SM the register budget is set for: at 7 (72 registers) a
+// 128,000-request launch is a single wave on 148 SMs; shared memory (18 KiB per block)
 // would allow 12.
 constexpr int kStepBlocksPerSM = 7;
 // Unroll factor of the scoring loop over the four 8-candidate groups: 2 keeps two window loads in

@@ -88,7 +88,9 @@ __device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg
     const uint8_t on = n.online[x];
     const int64_t queued = n.backlog[x];
     const uint32_t accept_util = n.accept_util_pm[x], accept_freq = n.accept_ppm[x];
-    const uint32_t u = ppm(draw(n, q, uint32_t(pick) >> 2, rg, kProbe).w[pick & 3]);
+    const Rnd4 y = draw(n, q, uint32_t(pick) >> 2, rg, kProbe);
+    const uint32_t sel = uint32_t(pick) & 3u;                            // selected without indexing: the words stay in registers
+    const uint32_t u = ppm(sel == 0 ? y.w[0] : sel == 1 ? y.w[1] : sel == 2 ? y.w[2] : y.w[3]);
     return on && cap != 0 && !util_at_least(cap, queued, n.util_window_ms, accept_util) && u < accept_freq;
 }
 
