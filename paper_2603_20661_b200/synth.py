@@ -281,6 +281,46 @@ def make_paper_setting(name: str, *, seed: int = 0, n_replicas: int = 64, offloa
     return Workload(name, st, peers, requests, batch=batch, gossip_every=1)
 
 
+SWEEP_AXES = ("stake", "accept", "offload")
+
+
+def make_policy_sweep(*, seed: int = 0, replicas_per_axis: int = 32, n_requests: int = 4000, batch: int = 500) -> Workload:
+    """The ablation on user-level policies as one batched run: a requester-only node 0 and four
+    providers (nodes 1-4), pure stake-proportional selection, and three groups of replicas that
+    differ in one policy each, every replica an independent repetition:
+
+      stake    stakes 1:2:3:4 (per-mille of credit 250, 500, 750, 1000), everybody accepts;
+      accept   equal stakes, acceptance frequencies 0.25, 0.5, 0.75, 1.0, at most three probes;
+      offload  requests arrive at the providers themselves, offloading frequencies 0.25 .. 1.0.
+
+    `wl.axis[r]` names the group of replica r (index into SWEEP_AXES)."""
+    rng = np.random.default_rng(np.random.PCG64(seed))
+    N, Rp, Q = 5, 3 * replicas_per_axis, n_requests
+    st = Settings(N, Rp, seed=seed, fanout_k=2, p_duel_ppm=100_000, max_probes=3, n_judges=1, flags=0)
+    shape = (Rp, N)
+    axis = np.repeat(np.arange(3), replicas_per_axis)
+    ramp = np.array([0, 0.25, 0.5, 0.75, 1.0])
+    cap = np.full(shape, 2000, np.uint32); cap[axis != 2, 0] = 0            # node 0 only issues requests
+    stake = np.full(shape, 1000, np.uint16); stake[axis == 0] = (1000 * ramp).astype(np.uint16); stake[axis == 0, 0] = 1000
+    accept = np.full(shape, 1_000_000, np.uint32); accept[axis == 1] = (1e6 * ramp).astype(np.uint32)
+    offload = np.full(shape, 1_000_000, np.uint32); offload[axis == 2] = (1e6 * ramp).astype(np.uint32)
+    peers = {
+        "cap_true_tok_s": cap, "quality_fx": _quality_to_fx(rng.random(shape)),
+        "credit0": np.full(shape, 10 ** 9, np.int64), "stake_pm": stake,
+        "offload_util_pm": np.zeros(shape, np.uint16), "accept_util_pm": np.full(shape, 1001, np.uint16),
+        "offload_ppm": offload, "accept_ppm": accept,
+        "misreport_mul": np.ones(shape, np.uint8), "prio_flag": np.zeros(shape, np.uint8), "online0": np.ones(shape, np.uint8),
+    }
+    origin = np.zeros((Rp, Q), np.uint32)
+    origin[axis == 2] = rng.integers(1, N, (replicas_per_axis, Q))
+    t = poisson_times_ms(rng, Q, 20.0)
+    rq = {"origin": origin, "t_ms": np.ascontiguousarray(np.broadcast_to(t, (Rp, Q))),
+          "len_in": _lengths(rng, (Rp, Q), 512.0), "len_out": _lengths(rng, (Rp, Q), 256.0)}
+    wl = Workload("policy_sweep", st, peers, rq, batch=batch, gossip_every=4)
+    wl.axis = axis
+    return wl
+
+
 def slice_replicas(wl: Workload, r0: int, r1: int) -> Workload:
     """The same workload restricted to replicas [r0, r1); randomness stays keyed
     by the global replica index through `replica_offset`."""
