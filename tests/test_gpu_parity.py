@@ -248,7 +248,7 @@ def test_fifo_queueing_matches_oracle(name, kw):
     assert o.stats_dict()["sum_latency_ms"] > 0
 
 
-@pytest.mark.parametrize("seed", range(int(os.environ.get("WWWS_FUZZ_SEEDS", "12"))))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("WWWS_FUZZ_SEEDS", "24"))))
 def test_random_configurations_match_oracle(seed):
     """Seeded random small networks: sizes, fanout, judges, probe budget, probabilities, all
     combinations of the behaviour flags, skewed ranks, misreporting, churn, stale initial views;
@@ -257,7 +257,8 @@ def test_random_configurations_match_oracle(seed):
     rng = np.random.default_rng(1000 + seed)
     N = int(rng.choice([2, 3, 9, 31, 32, 33, 64, 97, 200, 513]))
     Rp = int(rng.integers(1, 4))
-    Q, B = 360, int(rng.choice([1, 7, 60, 120]))
+    B = int(rng.choice([1, 7, 60, 120, 3500, 9000]))       # the large ones reach the 4-lane and the one-thread step kernels
+    Q = max(360, 3 * B)
     n_blk = (N + 31) // 32
     kw = dict(fanout_k=int(rng.integers(1, 5)), gossip_tries=int(rng.integers(1, 9)), max_probes=int(rng.integers(1, 8)),
               n_judges=int(rng.integers(1, 5)), p_duel_ppm=int(rng.choice([0, 100_000, 1_000_000])),
