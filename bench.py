@@ -280,7 +280,7 @@ def run_gpu(args):
                               "inputs smaller than L2 and not flushed: this workload is a launch-latency case, not a bandwidth one")},
             "clocks": clocks,
             "e2e": {"value": req_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / K, "entry": "wwws_step_host, pinned host buffers"},
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / K, "entry": "wwws_step_host, pinned host buffers (mapped: the kernels read requests from and write results to them)"},
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_request_path": roof_req,

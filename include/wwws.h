@@ -223,9 +223,12 @@ typedef struct {
     int32_t* exec_a; int32_t* exec_b; int32_t* judges; uint8_t* outcome; uint8_t* flags;
 } wwws_host_io;
 
-/* wwws_step with HOST buffers: copies the batch's request slices to the bound device arrays,
- * runs the step, copies the batch's results and the total counters back, and synchronises.
- * Host buffers should be pinned for full speed.  totals_out (HOST, one record) may be NULL. */
+/* wwws_step with HOST buffers; synchronises before it returns.  totals_out (HOST, one record) may be NULL.
+ * If all eight buffers are page-locked and mapped into the device's address space (cudaHostAlloc,
+ * cudaHostRegister) and exact queueing (WWWS_FLAG_FIFO) is off, the kernels read the batch's requests
+ * from, and write its results to, the host buffers directly; the bound device arrays are not touched.
+ * Otherwise the batch's request slices are copied to the bound device arrays, the step runs on
+ * those, and the batch's results are copied back.  Either way the total counters come back in totals_out. */
 wwws_status wwws_step_host(wwws_network* net, const wwws_host_io* io, uint64_t first, uint64_t count,
                            uint32_t now_ms, int do_gossip, int finalize, wwws_stats_t* totals_out);
 

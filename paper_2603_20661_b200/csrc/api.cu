@@ -361,6 +361,41 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
     if (wwws_status st = check_batch(n, first, count)) return st;
     if (!io || !io->origin || !io->len_in || !io->len_out || !io->exec_a || !io->exec_b || !io->judges || !io->outcome || !io->flags)
         return fail(n, WWWS_ERR_ARG, "a host buffer is NULL");
+    if (!(n->d.flags & 16u)) {
+        // Page-locked, mapped host buffers are read and written by the kernels themselves: no copies,
+        // and the result stores travel while the step runs.  (With exact queueing the results are
+        // read again by later kernels, which is better done from device memory.)
+        const void* host[8] = { io->origin, io->len_in, io->len_out, io->exec_a, io->exec_b, io->judges, io->outcome, io->flags };
+        void* dev[8];
+        bool direct = true;
+        for (int k = 0; k < 8 && direct; ++k) {
+            cudaPointerAttributes a;
+            if (cudaPointerGetAttributes(&a, host[k]) != cudaSuccess) { cudaGetLastError(); direct = false; }
+            else if (a.type != cudaMemoryTypeHost || !a.devicePointer) direct = false;
+            else dev[k] = a.devicePointer;
+        }
+        if (direct && (reinterpret_cast<uintptr_t>(dev[5]) & 15) == 0) {
+            Net& d = n->d;
+            const Net saved = d;
+            d.origin = static_cast<const uint32_t*>(dev[0]); d.len_in = static_cast<const uint16_t*>(dev[1]);
+            d.len_out = static_cast<const uint16_t*>(dev[2]);
+            d.exec_a = static_cast<int32_t*>(dev[3]); d.exec_b = static_cast<int32_t*>(dev[4]); d.judges = static_cast<int32_t*>(dev[5]);
+            d.outcome = static_cast<uint8_t*>(dev[6]); d.rflags = static_cast<uint8_t*>(dev[7]);
+            d.score_a = nullptr; d.score_sum = nullptr;
+            const wwws_status st = wwws_step(n, first, count, now_ms, do_gossip, finalize);
+            d.origin = saved.origin; d.len_in = saved.len_in; d.len_out = saved.len_out;
+            d.exec_a = saved.exec_a; d.exec_b = saved.exec_b; d.judges = saved.judges; d.outcome = saved.outcome; d.rflags = saved.rflags;
+            d.score_a = saved.score_a; d.score_sum = saved.score_sum;
+            if (st) return st;
+            if (totals_out) {
+                std::vector<wwws_stats_t> all(d.Rp + 1);
+                if (wwws_status st2 = wwws_stats(n, all.data())) return st2;
+                *totals_out = all[d.Rp];
+                return WWWS_OK;
+            }
+            return check_device_error(n);
+        }
+    }
     const Net& d = n->d;
     cudaStream_t s = n->stream;
     const size_t Q = d.Q, Rp = d.Rp, c = count;
