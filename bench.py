@@ -87,15 +87,17 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def step_args(wl, s):
+def step_args(wl, s, phase=0):
     """(first, count, now_ms, gossip) of global step s; the request stream is reused cyclically
-    while simulated time keeps growing."""
+    while simulated time keeps growing.  Gossip runs on the steps `phase`, `phase` + cadence, ...:
+    the timed steps start on a gossip step, so K timed steps hold ceil(K / cadence) rounds whatever
+    the warm-up count (never fewer than the workload's cadence asks for)."""
     n = wl.n_steps
     cyc, k = divmod(s, n)
     first = k * wl.batch
     cnt = min(wl.batch, wl.n_requests - first)
     t_end = int(wl.requests["t_ms"][0, -1]) + 1
-    return first, cnt, cyc * t_end + wl.step_now_ms(k), s % wl.gossip_every == 0
+    return first, cnt, cyc * t_end + wl.step_now_ms(k), (s - phase) % wl.gossip_every == 0
 
 
 def algorithmic_bytes(wl, stats_delta):
@@ -147,7 +149,8 @@ def run_gpu(args):
     W, K = args.warmup, args.steps
     s = 0
     for _ in range(W):
-        net.step(*step_args(wl, s)); s += 1
+        f, c, now, g = step_args(wl, s, W)
+        net.step(f, c, now, g or s == 0); s += 1        # a gossip round in the warm-up whatever the phase
     stats0 = net.stats()[-1].copy()
     launches0 = net.kernel_launches()
 
@@ -160,7 +163,7 @@ def run_gpu(args):
     barrier()
     ev0.record()
     for _ in range(K):
-        net.step(*step_args(wl, s)); s += 1
+        net.step(*step_args(wl, s, W)); s += 1
     ev1.record()
     barrier()
     ms = reduce_max(ev0.elapsed_time(ev1))
@@ -174,7 +177,7 @@ def run_gpu(args):
     barrier()
     ev0.record()
     for _ in range(K):
-        net.step(*step_args(wl, s)); s += 1
+        net.step(*step_args(wl, s, W)); s += 1
     ev1.record()
     barrier()
     ms_repeat = reduce_max(ev0.elapsed_time(ev1))
@@ -183,7 +186,7 @@ def run_gpu(args):
     net.profile(True)
     stats_b0 = net.stats()[-1].copy()
     for _ in range(K):
-        net.step(*step_args(wl, s)); s += 1
+        net.step(*step_args(wl, s, W)); s += 1
     prof = net.profile_read()
     net.profile(False)
     clocks = sampler.stop() if sampler else None     # sampled over region A and its instrumented repeat
@@ -225,14 +228,14 @@ def run_gpu(args):
 
     # ---- region S: the same K steps through the six separate calls ------------------------------
     for _ in range(min(W, 3)):                 # first use of the separate kernels loads their code: keep that untimed
-        net.run_step(*step_args(wl, s)); s += 1
-    while s % wl.gossip_every:
-        net.step(*step_args(wl, s)); s += 1
+        net.run_step(*step_args(wl, s, W)); s += 1
+    while (s - W) % wl.gossip_every:
+        net.step(*step_args(wl, s, W)); s += 1
     stats_s0 = net.stats()[-1].copy()
     barrier()
     ev0.record()
     for _ in range(K):
-        net.run_step(*step_args(wl, s)); s += 1
+        net.run_step(*step_args(wl, s, W)); s += 1
     ev1.record()
     barrier()
     ms_six = reduce_max(ev0.elapsed_time(ev1))
@@ -251,14 +254,14 @@ def run_gpu(args):
           "outcome": torch.empty((Rp, Q), dtype=torch.uint8).pin_memory(),
           "flags": torch.empty((Rp, Q), dtype=torch.uint8).pin_memory()}
     for _ in range(min(W, 3)):
-        net.step_host(io, *step_args(wl, s)); s += 1
-    while s % wl.gossip_every:                 # start the timed steps on a gossip step, as region A did
-        net.step_host(io, *step_args(wl, s)); s += 1
+        net.step_host(io, *step_args(wl, s, W)); s += 1
+    while (s - W) % wl.gossip_every:           # start the timed steps on a gossip step, as region A did
+        net.step_host(io, *step_args(wl, s, W)); s += 1
     stats_c0 = net.stats()[-1].copy()
     barrier()
     ev0.record()
     for _ in range(K):
-        tot = net.step_host(io, *step_args(wl, s)); s += 1
+        tot = net.step_host(io, *step_args(wl, s, W)); s += 1
     ev1.record()
     barrier()
     ms_e2e = reduce_max(ev0.elapsed_time(ev1))
@@ -273,7 +276,7 @@ def run_gpu(args):
             "ms_per_step": ms / K, "ms_per_step_repeat": ms_repeat / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u64 views, i64 ledgers, fp32 scores", "data": "synthetic",
             "config": {"workload": args.workload, "n_peers": st.n_peers, "n_replicas_per_gpu": Rp,
-                       "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "flags": st.flags, "gossip_every": wl.gossip_every,
+                       "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "flags": st.flags, "gossip_every": wl.gossip_every, "gossip_phase": "first timed step",
                        "fanout_k": st.fanout_k, "entry": "wwws_step (fused dispatch+duel+settle)",
                        "l2": ("inputs larger than L2 (view buffers %.1f GB per GPU)" % (2 * 8 * st.n_peers ** 2 * Rp / 1e9)
                               if 2 * 8 * st.n_peers ** 2 * Rp > 126e6 else
@@ -307,14 +310,14 @@ def oracle_run(workload, seed, steps, warmup, replicas=1, first_replica=0):
     o.bind_requests(wl.requests)
     s = 0
     for _ in range(warmup):
-        f, c, now, g = step_args(wl, s); o.run_step(f, c, now, g); s += 1
+        f, c, now, g = step_args(wl, s, warmup); o.run_step(f, c, now, g); s += 1
     n0 = o.stats_dict()["n_requests"]
     t0 = time.perf_counter()
     for _ in range(steps):
-        f, c, now, g = step_args(wl, s); o.run_step(f, c, now, g); s += 1
+        f, c, now, g = step_args(wl, s, warmup); o.run_step(f, c, now, g); s += 1
     dt = time.perf_counter() - t0
     n = o.stats_dict()["n_requests"] - n0
-    rounds = sum(1 for k in range(warmup, warmup + steps) if k % wl.gossip_every == 0)
+    rounds = sum(1 for k in range(steps) if k % wl.gossip_every == 0)
     desc = (f"{replicas} replica(s) of {workload}, {steps} steps of {wl.batch} requests with {rounds} gossip round(s), "
             f"single thread")
     o.close()
