@@ -5,6 +5,8 @@ benchmark times).  Replicas are independent and keyed by their global index, so 
 of the full run can be checked completely against the oracle run on that replica alone:
 every result record, every per-peer table, the counters, and sampled rows of its view matrix.
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -53,4 +55,28 @@ def test_one_replica_of_the_full_run_matches_the_oracle(name, replica, steps):
     dec = np.isin(rg["outcome"][:, :upto], (1, 2, 3))
     assert np.all(rg["exec_b"][:, :upto][dec] >= 0) and np.all(rg["exec_b"][:, :upto][~dec] == -1)
     assert o.error() == 0
+    g.close()
+
+
+@pytest.mark.skipif(os.environ.get("WWWS_MAX_SIZE") != "1",
+                    reason="the oracle needs over a minute and about 100 GB of host memory at 65,535 peers: set WWWS_MAX_SIZE=1")
+@pytest.mark.parametrize("n_peers", [32768, 65535])
+def test_largest_networks_match_the_oracle(n_peers):
+    """The maximum peer count (65,535: the narrowest view panels, a ragged last candidate block,
+    34 GB per view buffer) and half of it, one replica, two gossip rounds with churn and three
+    batches: tables, results, counters and the whole view matrix."""
+    from paper_2603_20661_b200.binding import Network
+    from tests.helpers import assert_same_state
+    wl = synth.make_workload("adversarial16k", n_replicas=1, n_requests=3000, n_peers=n_peers)
+    wl.settings.p_leave_ppm = wl.settings.p_join_ppm = 50_000
+    g = Network(wl.settings, wl.peers, wl.batch); g.bind_requests(wl.requests)
+    o = Oracle(wl.settings, wl.peers); o.bind_requests(wl.requests)
+    for s in range(3):
+        g.step(s * wl.batch, wl.batch, wl.step_now_ms(s), s < 2)
+        o.run_step(s * wl.batch, wl.batch, wl.step_now_ms(s), s < 2)
+    assert_same_state(g, o, f"{n_peers} peers", upto=3 * wl.batch, views=False)
+    ov = o.view()[0]
+    for r0 in range(0, n_peers, 4096):                        # block by block: never two full copies at once
+        a = g.view_rows(0, r0, min(4096, n_peers - r0))
+        assert np.array_equal(a, ov[r0:r0 + a.shape[0]]), f"view rows from {r0} differ"
     g.close()
