@@ -23,9 +23,11 @@
  *   duel-and-judge     closed-form win probabilities, Q_i of Assumption 3,
  *                      extra-request count identity N*alpha*p_d*(1+k)
  *   settlement         exact conservation of total credit, Lemma 1 mean payoff
- *   advance_time       parity unpinned: the drain/priority-window model is a
- *                      reading (the paper gives no formula); hand cases only
- *   latency/SLO (S4)   parity unpinned for the same reason; hand cases only
+ *   advance_time,      the queue model is a reading (the paper gives no formula); its
+ *   latency/SLO (S4)   arithmetic is pinned to Lindley's recursion for the unfinished work
+ *                      of a first-come-first-served server with batch arrivals, on random
+ *                      job sizes and gaps; the priority-window halving of capacity stays
+ *                      "parity unpinned": hand cases only
  *
  * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
  */
