@@ -222,3 +222,31 @@ def test_push_pull_exchange_is_symmetric_and_faster():
                 t_conv = t
         rounds[flags] = (t_conv, stale)
     assert rounds[8][1] < rounds[0][1], rounds       # steady-state staleness is lower with push-pull
+
+
+def test_partner_choice_is_uniform_and_slots_are_independent():
+    """After the first round of a fresh network, node p knows the new version of node i exactly when
+    i pulled p (the hello; pulled rows are old ones), so the view shows who pulled whom.  Every slot
+    picks uniformly among the other N - 1 peers, independently of the other slots:
+    P(i pulls p) = 1 - (1 - 1/(N-1))^k for every ordered pair, and the number of distinct partners
+    of a node has the occupancy distribution of k balls in N - 1 boxes."""
+    from tests.helpers import chi2_ok
+    N, k, Rp = 9, 3, 600
+    st, pa, _ = make_net(N, n_replicas=Rp, fanout_k=k, gossip_tries=8, seed=11)
+    o = Oracle(st, pa)
+    v0 = int(entry_ver(o.view()[0, 0, 0]))
+    o.gossip_round()
+    pulled = entry_ver(o.view()) == v0 + 1                       # [replica, p, i]: p knows i's new entry
+    idx = np.arange(N)
+    assert pulled[:, idx, idx].all()
+    pulled[:, idx, idx] = False
+    pairs = pulled.sum(0)[~np.eye(N, dtype=bool)]                # 72 ordered pairs, each Binomial(Rp, P)
+    P = 1 - (1 - 1 / (N - 1)) ** k
+    stat = float(((pairs - Rp * P) ** 2 / (Rp * P * (1 - P))).sum())
+    assert stat < 72 + 5 * np.sqrt(2 * 72), stat
+    # distinct partners per node: 1, 2 or 3 of 8 boxes
+    distinct = pulled.sum(1).ravel()                             # per (replica, i): how many p it pulled
+    m = N - 1
+    exp = np.array([m * 1, m * (m - 1) * 3, m * (m - 1) * (m - 2)], float) / m ** 3
+    ok, s2, _ = chi2_ok(np.bincount(distinct, minlength=4)[1:], distinct.size * exp)
+    assert ok, s2
