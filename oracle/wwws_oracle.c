@@ -16,8 +16,10 @@
  * Pins (tests that tie this file to something other than itself):
  *   philox4x32_10      published known-answer vectors of the generator
  *   merge / gossip     semilattice laws, monotone versions, convergence to the
- *                      column-wise maximum, detection of departed peers
- *   dispatch           first-pick frequency = s_i / sum s_j (Assumption 3),
+ *                      column-wise maximum, detection of departed peers, partner
+ *                      choice uniform and independent across slots
+ *   dispatch           candidate block follows the rank distribution,
+ *                      first-pick frequency = s_i / sum s_j (Assumption 3),
  *                      interval check with big integers, Plackett-Luce order
  *                      probabilities by enumeration, stake 1:2:3:4 scenario
  *   duel-and-judge     closed-form win probabilities, Q_i of Assumption 3,

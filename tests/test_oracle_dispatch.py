@@ -310,3 +310,32 @@ def test_greedy_rule_takes_the_best_weight_then_the_next():
         o3 = Oracle(st3, pa3); o3.bind_requests(rq3)
         o3.dispatch_batch(0, 4)
         assert np.all(o3.results()["exec_a"][0] == 1) and np.all((o3.results()["flags"][0] & 1) == flagged)
+
+
+def test_candidate_block_follows_the_rank_distribution():
+    """D3: the candidate window is the block `rank` places after the origin's own block on the id
+    ring; the rank is uniform, or drawn from a supplied distribution (Zipf(1.1) in config 3).
+    Equal stakes, everybody accepts, so the executor is uniform inside the chosen block."""
+    from paper_2603_20661_b200 import synth
+    N, Q, origin = 160, 60_000, 70                                # five blocks of 32; the origin sits in block 2
+    for cdf, law in ((None, np.full(5, 0.2)),
+                     (synth.zipf_rank_cdf(5, 1.1), (1 / np.arange(1, 6) ** 1.1) / (1 / np.arange(1, 6) ** 1.1).sum()),
+                     (synth.zipf_rank_cdf(3, 1.1), np.r_[(1 / np.arange(1, 4) ** 1.1) / (1 / np.arange(1, 4) ** 1.1).sum(), 0, 0])):
+        kw = {} if cdf is None else {"rank_cdf": cdf}
+        st, pa, rq = make_net(N, n_requests=Q, seed=21, flags=0, p_duel_ppm=0, origin=np.full(Q, origin, np.uint32),
+                              peers={"cap_true_tok_s": np.where(np.arange(N) == origin, 0, 2000), "credit0": 10 ** 9}, **kw)
+        o = Oracle(st, pa); o.bind_requests(rq)
+        o.dispatch_batch(0, Q)
+        ex = o.results()["exec_a"][0]
+        assert ex.min() >= 0 and np.all(ex != origin)
+        by_rank = np.bincount((ex // 32 - origin // 32) % 5, minlength=5)      # rank 0 = the origin's own block
+        ok, stat, _ = chi2_ok(by_rank, Q * law)
+        assert ok, (by_rank, Q * law, stat)
+        # inside a block: uniform over its eligible peers (31 in the origin's block, 32 elsewhere)
+        for blk in range(5):
+            cnt = np.bincount(ex[ex // 32 == blk] - 32 * blk, minlength=32)
+            if cnt.sum() == 0:
+                continue
+            elig = np.array([32 * blk + c != origin for c in range(32)])
+            ok, stat, _ = chi2_ok(cnt, cnt.sum() * elig / elig.sum())
+            assert ok, (blk, stat)
