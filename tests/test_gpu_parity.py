@@ -298,6 +298,25 @@ def test_random_configurations_match_oracle(seed):
     g.close()
 
 
+def test_many_replicas_of_a_tiny_network_match_oracle():
+    """20,000 replicas of a 3-peer network (the replica axis is a grid dimension of every kernel):
+    gossip, a 4-lane launch (one request per replica) and a one-thread launch (three per replica)."""
+    from paper_2603_20661_b200.binding import Network
+    Rp, N, Q = 20_000, 3, 4
+    rng = np.random.default_rng(17)
+    st, pa, rq = make_net(N, Rp, Q, seed=9, fanout_k=2, p_duel_ppm=500_000, n_judges=1, p_leave_ppm=50_000, p_join_ppm=300_000,
+                          origin=rng.integers(0, N, (Rp, Q)),
+                          peers={"cap_true_tok_s": rng.integers(0, 4000, (Rp, N)), "quality_fx": rng.integers(0, 2 ** 32, (Rp, N), dtype=np.uint64),
+                                 "accept_ppm": rng.integers(0, 1_000_001, (Rp, N))})
+    g = Network(st, pa, 3); g.bind_requests(rq)
+    o = Oracle(st, pa); o.bind_requests(rq)
+    for s, (first, cnt) in enumerate(((0, 1), (1, 3))):
+        g.step(first, cnt, 500 * (s + 1), True)
+        o.run_step(first, cnt, 500 * (s + 1), True)
+        assert_same_state(g, o, f"many replicas step {s}", upto=first + cnt)
+    g.close()
+
+
 def test_edge_cases_match_oracle():
     """Degenerate networks: two peers, a single request, everybody offline, nobody willing,
     requester-only origin, ragged window, duel probability one with tiny candidate sets."""
