@@ -71,11 +71,7 @@ __device__ __forceinline__ int pos_draw(const Net& n, Window& w, uint32_t lane)
 // D6: the drawn candidate answers by its true state and its own accept policy.
 __device__ __forceinline__ bool probe(const Net& n, const Window& w, int pick)
 {
-    const size_t x = size_t(w.r) * n.N + kWin * w.blk + pick;
-    const uint32_t cap = n.cap_eff[x];
-    if (!n.online[x] || cap == 0) return false;
-    if (util_at_least(cap, n.backlog[x], n.util_window_ms, n.accept_util_pm[x])) return false;
-    return ppm(draw(n, w.q, uint32_t(pick) >> 2, w.rg, kProbe).w[pick & 3]) < n.accept_ppm[x];
+    return probe_peer(n, w.r, w.rg, w.q, w.blk, pick);
 }
 
 // Draw-and-probe until somebody accepts, the probe budget is spent or nobody is left.
