@@ -21,6 +21,8 @@
  *     conserved) set a device error word that the next synchronising call reports;
  *     no kernel traps.
  *   - A handle is not thread-safe.
+ *   - A network lives on the GPU that holds its workspace.  Every call makes that GPU current
+ *     while it runs and restores the caller's device before it returns.
  *   - All randomness is Philox4x32-10 with key = seed and counter
  *     (index, slot, replica_offset + replica, stage + 256*attempt), so results do not
  *     depend on launch shapes or on how replicas are split over processes.
@@ -161,6 +163,7 @@ typedef enum {
     WWWS_T_D_CREDIT,     /* int64  pending */
     WWWS_T_D_WINS,       /* uint32 pending */
     WWWS_T_D_DUELS,      /* uint32 pending */
+    WWWS_T_BLK_SPENT,    /* int64  with WWWS_FLAG_FIFO: credits spent in the block that is still open */
     WWWS_T_COUNT
 } wwws_table;
 
@@ -292,12 +295,14 @@ const char* wwws_last_error(const wwws_network* net);
  * peer and replica) is taken from a fixed 1.5 MiB array inside the library image instead of
  * the workspace; every GPU that loads the library holds that array until the process exits.
  * The call itself allocates nothing on host or device paths of CUDA: no cudaMalloc, no
- * cudaFree, no allocating library routine.
+ * cudaFree, no allocating library routine.  Per-kernel timing (wwws_profile) creates CUDA
+ * events, so while it is switched on this call returns WWWS_ERR_STATE instead of running.
  *
  * Limit: n_replicas * n_peers <= 65536; larger networks get WWWS_ERR_ARG and must use
  * wwws_gossip_round.  The first call on each device looks up the array's device address
- * (with that device current - call it with the network's device current, as for every
- * other call) and should be made before any stream capture begins.  All calls, from all
+ * (the call makes the network's device current for that, as every call of this library
+ * does) and should be made before any stream capture begins; threads that make that first
+ * call at the same time all find the same address.  All calls, from all
  * networks on a device, share the one array: two such rounds that overlap on the GPU (two
  * streams) race and give wrong views; run them one after another.  The array keeps the
  * previous round's contents; nothing in it has to start at zero, because each round

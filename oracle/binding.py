@@ -21,7 +21,7 @@ STAT_NAMES = ("n_requests", "n_local", "n_fallback_local", "n_dropped", "n_faile
               "n_duel_cancelled", "n_draw", "n_judge_evals", "n_probes", "n_near_boundary", "slo_met",
               "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest", "n_uncovered", "blocks_rejected")
 TABLES = ("online", "cap_eff", "backlog", "ver", "credit", "stake", "wins", "duels", "served", "served_local",
-          "d_credit", "d_wins", "d_duels")
+          "d_credit", "d_wins", "d_duels", "blk_spent")
 
 
 def build(force: bool = False) -> str:

@@ -25,11 +25,17 @@
  *   duel-and-judge     closed-form win probabilities, Q_i of Assumption 3,
  *                      extra-request count identity N*alpha*p_d*(1+k)
  *   settlement         exact conservation of total credit, Lemma 1 mean payoff
+ *   create             initial views: staleness recomputed from a second Philox written in
+ *                      the test (itself checked against the published vectors), uniform on
+ *                      0..init_stale_max by chi-square, diagonal current; offline bit,
+ *                      advertised capacity (saturation included) and queue field against the
+ *                      inputs; initial ledger and stake (tests/test_oracle_create.py)
  *   advance_time,      the queue model is a reading (the paper gives no formula); its
  *   latency/SLO (S4)   arithmetic is pinned to Lindley's recursion for the unfinished work
  *                      of a first-come-first-served server with batch arrivals, on random
- *                      job sizes and gaps; the priority-window halving of capacity stays
- *                      "parity unpinned": hand cases only
+ *                      job sizes and gaps; the priority window (half rate while active) is
+ *                      recomputed peer by peer and window by window from the second Philox,
+ *                      plus hand cases and the active-window frequency
  *
  * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
  */
@@ -693,7 +699,7 @@ const float *orc_score_sum(const orc_net *n) { return n->score_sum; }
 
 /* copy one per-peer table, widened to int64, into out[Rp*N] */
 enum { T_ONLINE, T_CAP_EFF, T_BACKLOG, T_VER, T_CREDIT, T_STAKE, T_WINS, T_DUELS, T_SERVED, T_SERVED_LOCAL,
-       T_D_CREDIT, T_D_WINS, T_D_DUELS };
+       T_D_CREDIT, T_D_WINS, T_D_DUELS, T_BLK_SPENT };
 int orc_table(const orc_net *n, int which, int64_t *out)
 {
     size_t NP = (size_t)n->Rp * n->N;
@@ -713,6 +719,7 @@ int orc_table(const orc_net *n, int which, int64_t *out)
         case T_D_CREDIT: out[x] = p->d_credit; break;
         case T_D_WINS: out[x] = p->d_wins; break;
         case T_D_DUELS: out[x] = p->d_duels; break;
+        case T_BLK_SPENT: out[x] = p->blk_spent; break;
         default: return 1;
         }
     }

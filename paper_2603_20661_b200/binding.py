@@ -24,7 +24,7 @@ STAT_NAMES = ("n_requests", "n_local", "n_fallback_local", "n_dropped", "n_faile
 TABLES = {"online": (0, np.uint8), "cap_eff": (1, np.uint32), "backlog": (2, np.int64), "ver": (3, np.uint32),
           "credit": (4, np.int64), "stake": (5, np.int64), "wins": (6, np.uint32), "duels": (7, np.uint32),
           "served": (8, np.uint64), "served_local": (9, np.uint64), "d_credit": (10, np.int64),
-          "d_wins": (11, np.uint32), "d_duels": (12, np.uint32)}
+          "d_wins": (11, np.uint32), "d_duels": (12, np.uint32), "blk_spent": (13, np.int64)}
 EXPORTS = ("wwws_workspace_bytes", "wwws_create_network", "wwws_destroy_network", "wwws_bind_requests",
            "wwws_advance_time", "wwws_gossip_round", "wwws_dispatch_batch", "wwws_duel_judge", "wwws_settle_credits",
            "wwws_step", "wwws_step_host", "wwws_stats", "wwws_export_table", "wwws_import_table",

@@ -1,4 +1,5 @@
 // C-ABI of the wwws library: argument checks, workspace layout, call ordering, copies.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -16,6 +17,7 @@ struct wwws_network {
     Net d;                       // device pointers and scalars
     wwws_config cfg;
     cudaStream_t stream;
+    int device;                  // ordinal of the GPU that holds the workspace; every call runs there
     uint8_t* ws; uint64_t ws_bytes;
     uint32_t t_last_ms, round;
     int phase;                   // 0 idle, 1 dispatched, 2 judged
@@ -44,6 +46,24 @@ wwws_status fail(wwws_network* n, wwws_status st, const std::string& msg)
         cudaError_t e_ = (call);                                                                 \
         if (e_ != cudaSuccess) return fail(net, WWWS_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
     } while (0)
+
+// Makes the network's GPU current for the duration of a call and puts the caller's back
+// afterwards: a handle works whatever device the calling thread has selected.
+struct DeviceScope {
+    int prev = -1; bool switched = false; cudaError_t err;
+    explicit DeviceScope(int want)
+    {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != want) { err = cudaSetDevice(want); switched = err == cudaSuccess; }
+    }
+    ~DeviceScope() { if (switched) cudaSetDevice(prev); }
+    DeviceScope(const DeviceScope&) = delete;
+    DeviceScope& operator=(const DeviceScope&) = delete;
+};
+#define ON_DEVICE(net)                                                                           \
+    DeviceScope device_scope_((net)->device);                                                    \
+    if (device_scope_.err != cudaSuccess)                                                        \
+        return fail(net, WWWS_ERR_CUDA, std::string("selecting the network's device: ") + cudaGetErrorString(device_scope_.err))
 
 const char* check_config(const wwws_config* c)
 {
@@ -177,12 +197,25 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
         if (init->misreport_mul[x] == 0) return fail(nullptr, WWWS_ERR_ARG, "misreport_mul must be >= 1");
     }
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return fail(nullptr, WWWS_ERR_ALLOC, "workspace is NULL or not 256-byte aligned");
+    // the GPU that holds the workspace is the network's GPU, whatever device is current now or later
+    cudaPointerAttributes wa;
+    if (cudaError_t e = cudaPointerGetAttributes(&wa, workspace); e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(nullptr, WWWS_ERR_CUDA, std::string("cudaPointerGetAttributes(workspace): ") + cudaGetErrorString(e));
+    }
+    if (wa.type != cudaMemoryTypeDevice && wa.type != cudaMemoryTypeManaged)
+        return fail(nullptr, WWWS_ERR_ARG, "workspace is not device memory");
     Carver cv{ static_cast<uint8_t*>(workspace), 0 };
     wwws_network* n = new (std::nothrow) wwws_network();
     if (!n) return fail(nullptr, WWWS_ERR_ALLOC, "host allocation failed");
+    n->device = wa.device;
+    struct Guard { wwws_network* n; ~Guard() { delete n; } } guard{ n };     // freed on every failure below
+    DeviceScope device_scope_(n->device);
+    if (device_scope_.err != cudaSuccess)
+        return fail(nullptr, WWWS_ERR_CUDA, std::string("selecting the workspace's device: ") + cudaGetErrorString(device_scope_.err));
     Staging sg{};
     carve(*cfg, cv, n->d, sg);
-    if (cv.off > workspace_bytes) { delete n; return fail(nullptr, WWWS_ERR_ALLOC, "workspace too small"); }
+    if (cv.off > workspace_bytes) return fail(nullptr, WWWS_ERR_ALLOC, "workspace too small");
     n->cfg = *cfg; n->cfg.rank_cdf = nullptr;
     n->stream = static_cast<cudaStream_t>(cuda_stream);
     n->ws = static_cast<uint8_t*>(workspace); n->ws_bytes = workspace_bytes;
@@ -202,13 +235,12 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
 
     wwws_network::TableInfo ti[WWWS_T_COUNT] = {
         { d.online, 1 }, { d.cap_eff, 4 }, { d.backlog, 8 }, { d.ver, 4 }, { d.credit, 8 }, { d.stake, 8 }, { d.wins, 4 },
-        { d.duels, 4 }, { d.served, 8 }, { d.served_local, 8 }, { d.d_credit, 8 }, { d.d_wins, 4 }, { d.d_duels, 4 } };
+        { d.duels, 4 }, { d.served, 8 }, { d.served_local, 8 }, { d.d_credit, 8 }, { d.d_wins, 4 }, { d.d_duels, 4 },
+        { d.blk_spent, 8 } };
     memcpy(n->tables, ti, sizeof ti);
 
     cudaStream_t s = n->stream;
 #define H2D(dst, src, T) CUDA_TRY(nullptr, cudaMemcpyAsync(const_cast<T*>(dst), src, NP * sizeof(T), cudaMemcpyHostToDevice, s))
-    // on failure below the handle leaks nothing but itself; free it before returning
-    struct Guard { wwws_network* n; ~Guard() { delete n; } } guard{ n };
     H2D(d.cap_true, init->cap_true_tok_s, uint32_t); H2D(d.quality, init->quality_fx, uint32_t);
     H2D(d.stake_pm, init->stake_pm, uint16_t); H2D(d.offload_util_pm, init->offload_util_pm, uint16_t);
     H2D(d.accept_util_pm, init->accept_util_pm, uint16_t);
@@ -246,7 +278,10 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
 wwws_status wwws_destroy_network(wwws_network* n)
 {
     if (!n) return WWWS_OK;
-    cudaStreamSynchronize(n->stream);
+    {
+        DeviceScope scope(n->device);
+        cudaStreamSynchronize(n->stream);
+    }
     delete n;
     return WWWS_OK;
 }
@@ -273,6 +308,7 @@ wwws_status wwws_advance_time(wwws_network* n, uint32_t now_ms)
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (now_ms < n->t_last_ms) return fail(n, WWWS_ERR_ARG, "time must not go back");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "advance_time inside a batch");
+    ON_DEVICE(n);
     launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx());
     n->t_last_ms = now_ms;
     return launch_status(n, "advance_time");
@@ -282,6 +318,7 @@ wwws_status wwws_gossip_round(wwws_network* n)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "gossip_round inside a batch");
+    ON_DEVICE(n);
     launch_gossip(n->d, n->round, n->ctx());
     std::swap(n->d.view, n->d.view_new);
     n->round += 1;
@@ -311,6 +348,7 @@ static bool threads_for(const wwws_network* n, uint64_t count)
 wwws_status wwws_dispatch_batch(wwws_network* n, uint64_t first, uint64_t count)
 {
     if (wwws_status st = check_batch(n, first, count)) return st;
+    ON_DEVICE(n);
     if (threads_for(n, count)) launch_dispatch_threads(n->d, first, uint32_t(count), n->ctx());
     else launch_dispatch(n->d, first, uint32_t(count), n->ctx());
     n->batch_first = first; n->batch_count = uint32_t(count); n->phase = 1;
@@ -321,6 +359,7 @@ wwws_status wwws_duel_judge(wwws_network* n)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 1) return fail(n, WWWS_ERR_STATE, "duel_judge must follow dispatch_batch");
+    ON_DEVICE(n);
     if (threads_for(n, n->batch_count)) launch_duel_threads(n->d, n->batch_first, n->batch_count, n->ctx());
     else launch_duel(n->d, n->batch_first, n->batch_count, n->ctx());
     n->phase = 2;
@@ -331,6 +370,7 @@ wwws_status wwws_settle_credits(wwws_network* n, int finalize)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 2) return fail(n, WWWS_ERR_STATE, "settle_credits must follow duel_judge");
+    ON_DEVICE(n);
     launch_settle(n->d, n->batch_first, n->batch_count, n->ctx());
     if (n->d.flags & 16u) launch_fifo(n->d, n->batch_first, n->batch_count, n->ctx());
     launch_fold(n->d, finalize != 0, n->ctx());
@@ -342,6 +382,7 @@ wwws_status wwws_step(wwws_network* n, uint64_t first, uint64_t count, uint32_t 
 {
     if (wwws_status st = check_batch(n, first, count)) return st;
     if (now_ms < n->t_last_ms) return fail(n, WWWS_ERR_ARG, "time must not go back");
+    ON_DEVICE(n);
     launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx());
     n->t_last_ms = now_ms;
     if (do_gossip) {
@@ -361,6 +402,7 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
     if (wwws_status st = check_batch(n, first, count)) return st;
     if (!io || !io->origin || !io->len_in || !io->len_out || !io->exec_a || !io->exec_b || !io->judges || !io->outcome || !io->flags)
         return fail(n, WWWS_ERR_ARG, "a host buffer is NULL");
+    ON_DEVICE(n);
     if (!(n->d.flags & 16u)) {
         // Page-locked, mapped host buffers are read and written by the kernels themselves: no copies,
         // and the result stores travel while the step runs.  (With exact queueing the results are
@@ -424,6 +466,7 @@ wwws_status wwws_stats(wwws_network* n, wwws_stats_t* host_out)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (!host_out) return fail(n, WWWS_ERR_ARG, "host_out is NULL");
+    ON_DEVICE(n);
     launch_credit_total(n->d, n->ctx());
     if (wwws_status st = launch_status(n, "stats")) return st;
     CUDA_TRY(n, cudaMemcpyAsync(host_out, n->d.stats, uint64_t(n->d.Rp) * sizeof(wwws_stats_t), cudaMemcpyDeviceToHost, n->stream));
@@ -443,6 +486,7 @@ wwws_status wwws_export_table(wwws_network* n, wwws_table t, void* host_dst, uin
     if (!host_dst || int(t) < 0 || t >= WWWS_T_COUNT) return fail(n, WWWS_ERR_ARG, "bad table or NULL destination");
     const uint64_t need = uint64_t(n->d.N) * n->d.Rp * n->tables[t].elem;
     if (bytes != need) return fail(n, WWWS_ERR_ARG, "bytes does not match the table size");
+    ON_DEVICE(n);
     CUDA_TRY(n, cudaMemcpyAsync(host_dst, n->tables[t].ptr, need, cudaMemcpyDeviceToHost, n->stream));
     return check_device_error(n);
 }
@@ -454,6 +498,7 @@ wwws_status wwws_import_table(wwws_network* n, wwws_table t, const void* host_sr
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
     const uint64_t need = uint64_t(n->d.N) * n->d.Rp * n->tables[t].elem;
     if (bytes != need) return fail(n, WWWS_ERR_ARG, "bytes does not match the table size");
+    ON_DEVICE(n);
     CUDA_TRY(n, cudaMemcpyAsync(n->tables[t].ptr, host_src, need, cudaMemcpyHostToDevice, n->stream));
     if (t == WWWS_T_CREDIT || t == WWWS_T_WINS || t == WWWS_T_DUELS) launch_rederive(n->d, n->ctx());
     CUDA_TRY(n, cudaStreamSynchronize(n->stream));
@@ -465,6 +510,7 @@ wwws_status wwws_export_view_rows(wwws_network* n, uint32_t replica, uint32_t ro
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (!host_dst) return fail(n, WWWS_ERR_ARG, "host_dst is NULL");
     if (replica >= n->d.Rp || uint64_t(row_first) + n_rows > n->d.N) return fail(n, WWWS_ERR_ARG, "rows out of range");
+    ON_DEVICE(n);
     if (n_rows == 0) return WWWS_OK;
     const uint64_t* src = n->d.view + (uint64_t(replica) * n->d.N + row_first) * n->d.ld;
     CUDA_TRY(n, cudaMemcpy2DAsync(host_dst, n->d.N * 8ull, src, n->d.ld * 8ull, n->d.N * 8ull, n_rows, cudaMemcpyDeviceToHost, n->stream));
@@ -477,6 +523,7 @@ wwws_status wwws_import_view_rows(wwws_network* n, uint32_t replica, uint32_t ro
     if (!host_src) return fail(n, WWWS_ERR_ARG, "host_src is NULL");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
     if (replica >= n->d.Rp || uint64_t(row_first) + n_rows > n->d.N) return fail(n, WWWS_ERR_ARG, "rows out of range");
+    ON_DEVICE(n);
     if (n_rows == 0) return WWWS_OK;
     uint64_t* dst = n->d.view + (uint64_t(replica) * n->d.N + row_first) * n->d.ld;
     CUDA_TRY(n, cudaMemcpy2DAsync(dst, n->d.ld * 8ull, host_src, n->d.N * 8ull, n->d.N * 8ull, n_rows, cudaMemcpyHostToDevice, n->stream));
@@ -505,6 +552,7 @@ wwws_status wwws_import_stats(wwws_network* n, const wwws_stats_t* host_src)
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (!host_src) return fail(n, WWWS_ERR_ARG, "host_src is NULL");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
+    ON_DEVICE(n);
     CUDA_TRY(n, cudaMemcpyAsync(n->d.stats, host_src, uint64_t(n->d.Rp) * sizeof(wwws_stats_t), cudaMemcpyHostToDevice, n->stream));
     CUDA_TRY(n, cudaStreamSynchronize(n->stream));
     return WWWS_OK;
@@ -528,6 +576,7 @@ uint64_t wwws_kernel_launches(const wwws_network* n) { return n ? n->launches : 
 wwws_status wwws_profile(wwws_network* n, int enable)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
+    ON_DEVICE(n);
     n->prof.reset();
     n->prof.enabled = enable != 0;
     return WWWS_OK;
@@ -537,6 +586,7 @@ wwws_status wwws_profile_read(wwws_network* n, double* ms_out, uint64_t* count_o
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (!ms_out || !count_out) return fail(n, WWWS_ERR_ARG, "output array is NULL");
+    ON_DEVICE(n);
     n->prof.collect();
     for (int k = 0; k < kKernelCount; ++k) { ms_out[k] = n->prof.ms[k]; count_out[k] = n->prof.count[k]; }
     return WWWS_OK;
@@ -573,7 +623,8 @@ constexpr uint64_t kStaticPartnerBytes = kStaticPeers * 4 * sizeof(int32_t);
 static __device__ __align__(256) unsigned char g_gossip_scratch[kStaticSelfBytes + kStaticPartnerBytes];  // 1.5 MiB
 
 constexpr int kMaxDevices = 64;
-void* g_gossip_scratch_addr[kMaxDevices];                      // per device, filled on first use
+std::atomic<void*> g_gossip_scratch_addr[kMaxDevices];         // per device, filled on first use; handles on
+                                                               // several threads may resolve it at once (same value)
 
 }  // namespace
 
@@ -581,6 +632,7 @@ extern "C" wwws_status wwws_gossip_round_static(wwws_network* n)
 {
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "gossip_round inside a batch");
+    if (n->prof.enabled) return fail(n, WWWS_ERR_STATE, "per-kernel timing creates CUDA events: switch wwws_profile off for the round that allocates nothing");
     const uint64_t peers = uint64_t(n->d.N) * n->d.Rp;
     if (peers > kStaticPeers) {
         char buf[160];
@@ -588,17 +640,18 @@ extern "C" wwws_status wwws_gossip_round_static(wwws_network* n)
                  (unsigned long long)peers, (unsigned long long)kStaticPeers);
         return fail(n, WWWS_ERR_ARG, buf);
     }
-    int dev = -1;
-    CUDA_TRY(n, cudaGetDevice(&dev));
+    const int dev = n->device;
     if (dev < 0 || dev >= kMaxDevices) return fail(n, WWWS_ERR_ARG, "device ordinal beyond 63");
-    if (!g_gossip_scratch_addr[dev]) {
+    ON_DEVICE(n);
+    void* p = g_gossip_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!p) {
         // In host code the array's name is only a handle for the runtime; the address the
-        // kernels need comes from the runtime, for the device that is current now.
-        void* p = nullptr;
+        // kernels need comes from the runtime, for the device that is current now (the
+        // network's own, selected just above).
         CUDA_TRY(n, cudaGetSymbolAddress(&p, g_gossip_scratch));
-        g_gossip_scratch_addr[dev] = p;
+        g_gossip_scratch_addr[dev].store(p, std::memory_order_release);
     }
-    unsigned char* base = static_cast<unsigned char*>(g_gossip_scratch_addr[dev]);
+    unsigned char* base = static_cast<unsigned char*>(p);
     Net d = n->d;                                              // same network, scratch pointers redirected
     d.self_entry = reinterpret_cast<uint64_t*>(base);
     d.partner = reinterpret_cast<int32_t*>(base + kStaticSelfBytes);

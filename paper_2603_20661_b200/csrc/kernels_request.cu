@@ -223,7 +223,7 @@ __global__ void k_fifo_fill(Net n, uint32_t count)
     if (item.x < 0) return;
     const size_t px = size_t(r) * n.N + item.x;
     const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
-    // entry: (request, amount), bit 31 of the amount marks a payment (role 6) as opposed to queued work
+    // entry: (request, amount): tokens of queued work, or, with bit 31 set, the number of payments of R (role 6)
     n.fifo_list[size_t(r) * n.max_batch * 7 + n.in_off[px] + k] = make_uint2(slot / 7, uint32_t(item.y) | (slot % 7 == 6 ? 0x80000000u : 0u));
 }
 
@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
                 const uint2* mine = n.fifo_list + size_t(r) * n.max_batch * 7 + n.in_off[ox];
                 const uint32_t mlen = n.in_deg[ox];
                 long long spent = n.blk_spent[ox];
-                for (uint32_t j = 0; j < mlen; ++j) { const uint2 it = mine[j]; if (it.x < idx && (it.y >> 31)) spent += it.y & 0x7fffffffu; }
+                for (uint32_t j = 0; j < mlen; ++j) { const uint2 it = mine[j]; if (it.x < idx && (it.y >> 31)) spent += n.R * (long long)(it.y & 0x7fffffffu); }
                 const uint32_t oc = n.outcome[x];
                 const long long pay = n.R * ((oc >= 1 && oc <= 3) ? 2 : 1);
                 uncovered = n.credit[ox] - spent < pay;

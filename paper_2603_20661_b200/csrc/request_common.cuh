@@ -157,9 +157,10 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
         fifo_emit(n, r, bidx, 1, duel ? b : -1, li + lo);
 #pragma unroll
         for (int l = 0; l < 4; ++l) fifo_emit(n, r, bidx, 2 + l, duel ? jd[l] : -1, li + 2u * lo);
-        const uint32_t pay = uint32_t(n.R) * (duel ? 2u : 1u);
-        fifo_emit(n, r, bidx, 6, a >= 0 ? int(o) : -1, pay);
-        if (a >= 0) add64(&n.d_spent[size_t(r) * n.N + o], (long long)pay);
+        // the payment's slot carries the number of transactions of R (two for a duel); the amount stays 64-bit
+        const uint32_t n_pay = duel ? 2u : 1u;
+        fifo_emit(n, r, bidx, 6, a >= 0 ? int(o) : -1, n_pay);
+        if (a >= 0) add64(&n.d_spent[size_t(r) * n.N + o], n.R * (long long)n_pay);
     }
     const size_t base = size_t(r) * n.N;
     const uint64_t work = uint64_t(li) + lo;

@@ -77,7 +77,7 @@ def chi2_ok(obs, exp, z=5.0):
 # ---- GPU-vs-oracle comparison -----------------------------------------------------------------
 
 TABLE_NAMES = ("online", "cap_eff", "backlog", "ver", "credit", "stake", "wins", "duels", "served", "served_local",
-               "d_credit", "d_wins", "d_duels")
+               "d_credit", "d_wins", "d_duels", "blk_spent")
 
 
 def assert_same_state(gpu, orc, where, upto=None, views=True, scores=True, stats=True):

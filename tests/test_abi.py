@@ -67,6 +67,16 @@ def test_host_side_argument_checks():
     assert lib.wwws_create_network(C.byref(cfg4), C.byref(init), None, 0, None, C.byref(h)) == 1
     assert h.value is None
     assert lib.wwws_create_network(C.byref(cfg4), None, None, 0, None, C.byref(h)) == 1
+    # a workspace that is not device memory is refused before anything is built on it: the GPU that
+    # holds the workspace is the network's GPU, and every later call runs there whatever device is current
+    pa = {k: np.ascontiguousarray(np.broadcast_to(np.asarray(v), (2, 64)).astype(dt)) for (k, dt), v in
+          zip(binding.PEER_ORDER, (2000, 1 << 31, 10_000, 1000, 0, 1001, 10 ** 6, 10 ** 6, 1, 0, 1))}
+    for k, _ in binding.PEER_ORDER:
+        setattr(init, k, pa[k].ctypes.data)
+    host_ws = np.zeros(n.value + 256, np.uint8)
+    addr = (host_ws.ctypes.data + 255) & ~255
+    assert lib.wwws_create_network(C.byref(cfg4), C.byref(init), addr, n.value, None, C.byref(h)) in (1, 5)
+    assert h.value is None and len(lib.wwws_last_error(None)) > 0
     # null handles
     assert lib.wwws_gossip_round(None) == 1 and lib.wwws_dispatch_batch(None, 0, 1) == 1
     assert lib.wwws_gossip_round_static(None) == 1

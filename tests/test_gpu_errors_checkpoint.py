@@ -66,23 +66,31 @@ def test_version_overflow_is_reported():
     assert e.value.status == 4
 
 
-def test_checkpoint_resume_continues_bit_for_bit():
+@pytest.mark.parametrize("flags,cut", [(0, 3), (16, 2)], ids=["block_closed_at_the_cut", "exact_queueing_block_open_at_the_cut"])
+def test_checkpoint_resume_continues_bit_for_bit(flags, cut):
+    """Steps 0 and 2 finalize, step 1 does not: a cut after two steps leaves a block open, and with
+    exact queueing the credits spent inside it (table blk_spent) decide which later payments are covered."""
     from paper_2603_20661_b200.binding import Network
     wl = synth.make_workload("churn4k", n_replicas=2, n_requests=6000, n_peers=300)
     wl.settings.p_duel_ppm = 300_000
+    wl.settings.flags |= flags
+    if flags & 16:
+        wl.peers["credit0"][:] = 900              # a few payments per peer are covered, the rest are not
 
     def run(net, s0, s1):
         for s in range(s0, s1):
             net.step(s * wl.batch, wl.batch, wl.step_now_ms(s), s % 2 == 0, s % 3 != 1)
 
     a = Network(wl.settings, wl.peers, wl.batch); a.bind_requests(wl.requests)
-    run(a, 0, 3)
+    run(a, 0, cut)
     ck = a.checkpoint()
+    if flags & 16:
+        assert ck["tables"]["blk_spent"].any() and ck["tables"]["d_credit"].any()       # the cut is inside a block
     b = Network(wl.settings, wl.peers, wl.batch); b.bind_requests(wl.requests)
     b.restore(ck)
-    run(a, 3, 6); run(b, 3, 6)
+    run(a, cut, 6); run(b, cut, 6)
     ra, rb = a.results(), b.results()
-    lo, hi = 3 * wl.batch, 6 * wl.batch
+    lo, hi = cut * wl.batch, 6 * wl.batch
     for k in ("exec_a", "exec_b", "judges", "outcome", "flags"):
         assert np.array_equal(ra[k][:, lo:hi], rb[k][:, lo:hi]), k
     assert np.array_equal(a.view(), b.view()) and np.array_equal(a.stats(), b.stats())
@@ -90,3 +98,5 @@ def test_checkpoint_resume_continues_bit_for_bit():
     for k in ca["tables"]:
         assert np.array_equal(ca["tables"][k], cb["tables"][k]), k
     assert ca["clock"] == cb["clock"]
+    if flags & 16:
+        assert a.stats_dict()["n_uncovered"] > 0

@@ -346,6 +346,10 @@ def test_edge_cases_match_oracle():
     # exact queueing + in-block validation with a payer that runs out of covered credit
     cases.append(make_net(6, n_requests=300, seed=11, flags=3 | 16, p_duel_ppm=400_000, n_judges=2,
                           peers=requester_first(6, credit0=np.array([5_000, 10 ** 6, 10 ** 6, 10 ** 6, 10 ** 6, 10 ** 6]))))
+    # the same with rewards far beyond 32 bits: payments and in-block spending stay 64-bit throughout
+    cases.append(make_net(6, n_requests=300, seed=13, flags=3 | 16, p_duel_ppm=400_000, n_judges=2,
+                          reward_R=2 ** 33 + 5, reward_add=2 ** 20 + 1, penalty_P=2 ** 21 + 7,
+                          peers=requester_first(6, credit0=np.array([2 ** 39, 2 ** 36, 2 ** 36, 2 ** 35, 2 ** 40, 2 ** 34]))))
     for ci, (st, pa, rq) in enumerate(cases):
         g = Network(st, pa, 128); g.bind_requests(rq)
         o = Oracle(st, pa); o.bind_requests(rq)

@@ -9,7 +9,9 @@ array per GPU, and a failure here must not hide results of the other tests.
 import numpy as np
 import pytest
 
+from oracle import Oracle
 from paper_2603_20661_b200 import synth
+from tests.helpers import assert_same_state
 
 pytestmark = pytest.mark.gpu
 
@@ -24,17 +26,31 @@ def _evolved_network(wl):
     return net
 
 
-def test_static_round_equals_ordinary_round_twice_in_a_row():
+def _evolved_oracle(wl):
+    o = Oracle(wl.settings, wl.peers)
+    o.bind_requests(wl.requests)
+    for s in range(3):
+        o.run_step(s * wl.batch, wl.batch, wl.step_now_ms(s), s == 0)
+    return o
+
+
+@pytest.mark.parametrize("push_pull", [False, True], ids=["pull", "pairwise_exchange"])
+def test_static_round_equals_ordinary_round_twice_in_a_row(push_pull):
     wl = synth.make_workload("churn4k", n_replicas=3, n_requests=4000, n_peers=1100)
-    a, b = _evolved_network(wl), _evolved_network(wl)
+    if push_pull:
+        wl.settings.flags |= 8                # the partner lists in the built-in array also feed the reverse lists
+    a, b, o = _evolved_network(wl), _evolved_network(wl), _evolved_oracle(wl)
     assert np.array_equal(a.view(), b.view())
     for rnd in range(2):                      # second call reuses the array with the first call's contents in it
         a.gossip_round()
         b.gossip_round_static()
+        o.gossip_round()
         assert np.array_equal(a.view(), b.view()), f"round {rnd}: views differ"
         for t in ("online", "backlog", "ver"):
             assert np.array_equal(a.table(t), b.table(t)), f"round {rnd}: {t} differs"
         assert np.array_equal(a.stats(), b.stats()), f"round {rnd}: counters differ"
+        # and against the CPU oracle: every table, the whole view matrix, the counters
+        assert_same_state(b, o, f"static round {rnd}", upto=3 * wl.batch)
     # the networks stay interchangeable afterwards
     a.step(3 * wl.batch, wl.batch, wl.step_now_ms(3), True)
     b.step(3 * wl.batch, wl.batch, wl.step_now_ms(3), True)
