@@ -264,9 +264,15 @@ wwws_status wwws_import_stats(wwws_network* net, const wwws_stats_t* host_src);
 
 /* Tuning options; results never depend on them. */
 typedef enum {
-    WWWS_OPT_REQUEST_KERNEL = 0 /* implementation of wwws_dispatch_batch / wwws_duel_judge: 0 chosen by launch size
+    WWWS_OPT_REQUEST_KERNEL = 0,/* implementation of wwws_dispatch_batch / wwws_duel_judge: 0 chosen by launch size
                                    (default), 1 one warp per request (lane per candidate, warp-shuffle prefix sums),
                                    2 one thread per request (weights in shared memory, duels compacted per block) */
+    WWWS_OPT_STEP_KERNEL = 1,   /* implementation of wwws_step's fused kernel: 0 chosen by launch size (default),
+                                   1 eight lanes per request, 2 four lanes per request, 3 one thread per request,
+                                   4 streaming phases (a warp takes a run of requests through origin / score /
+                                   draw / vote / finish with full warps) */
+    WWWS_OPT_STREAM_RUN = 2     /* requests per warp of the streaming kernel: 0 chosen by launch size (default),
+                                   else a multiple of 32 */
 } wwws_option;
 wwws_status wwws_set_option(wwws_network* net, wwws_option option, int64_t value);
 

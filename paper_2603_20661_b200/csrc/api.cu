@@ -24,6 +24,8 @@ struct wwws_network {
     uint64_t batch_first; uint32_t batch_count;
     bool bound;
     int request_kernel;          // 0 by launch size, 1 warp per request, 2 thread per request
+    int step_kernel;             // fused step: 0 by launch size, 1/2 eight/four lanes per request, 3 one thread, 4 streaming phases
+    uint32_t stream_run;         // requests per warp of the streaming kernel, 0 = by launch size
     uint64_t launches;
     Profiler prof;
     std::string err;
@@ -124,7 +126,8 @@ void carve(const wwws_config& c, Carver& cv, Net& d, Staging& sg)
     d.served = cv.take<unsigned long long>(NP); d.served_local = cv.take<unsigned long long>(NP);
     d.d_credit = cv.take<long long>(NP); d.d_wins = cv.take<uint32_t>(NP); d.d_duels = cv.take<uint32_t>(NP);
     d.d_backlog = cv.take<long long>(NP);
-    d.w_led = cv.take<float>(NP);
+    d.w_led = cv.take<float>(Rp * ld);
+    d.gate = cv.take<uint64_t>(NP);
     d.self_entry = cv.take<uint64_t>(NP); d.partner = cv.take<int32_t>(NP * 4);
     d.in_deg = cv.take<uint32_t>(NP); d.in_off = cv.take<uint32_t>(NP); d.in_cursor = cv.take<uint32_t>(NP);
     d.pullers = cv.take<int32_t>(NP * 4);
@@ -266,6 +269,7 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
     CUDA_TRY(nullptr, cudaMemsetAsync(d.err, 0, 16, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.partner, 0xff, NP * 16, s));
     CUDA_TRY(nullptr, cudaMemsetAsync(d.in_deg, 0, NP * 4, s));
+    CUDA_TRY(nullptr, cudaMemsetAsync(d.w_led, 0, uint64_t(d.Rp) * d.ld * 4, s));   // padding columns stay 0
     launch_peer_init(d, sg.credit0, sg.online0, cfg->init_stale_max, n->ctx());
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return fail(nullptr, WWWS_ERR_CUDA, std::string("initialisation kernels: ") + cudaGetErrorString(e));
     // host staging (`tot`, the caller's arrays) must stay valid until the copies are done
@@ -390,7 +394,7 @@ wwws_status wwws_step(wwws_network* n, uint64_t first, uint64_t count, uint32_t 
         std::swap(n->d.view, n->d.view_new);
         n->round += 1;
     }
-    launch_step_fused(n->d, first, uint32_t(count), n->ctx());
+    launch_step_fused(n->d, first, uint32_t(count), n->ctx(), n->step_kernel, n->stream_run);
     if (n->d.flags & 16u) launch_fifo(n->d, first, uint32_t(count), n->ctx());
     launch_fold(n->d, finalize != 0, n->ctx());
     return launch_status(n, "step");
@@ -500,7 +504,8 @@ wwws_status wwws_import_table(wwws_network* n, wwws_table t, const void* host_sr
     if (bytes != need) return fail(n, WWWS_ERR_ARG, "bytes does not match the table size");
     ON_DEVICE(n);
     CUDA_TRY(n, cudaMemcpyAsync(n->tables[t].ptr, host_src, need, cudaMemcpyHostToDevice, n->stream));
-    if (t == WWWS_T_CREDIT || t == WWWS_T_WINS || t == WWWS_T_DUELS) launch_rederive(n->d, n->ctx());
+    if (t == WWWS_T_CREDIT || t == WWWS_T_WINS || t == WWWS_T_DUELS || t == WWWS_T_ONLINE || t == WWWS_T_CAP_EFF || t == WWWS_T_BACKLOG)
+        launch_rederive(n->d, n->ctx());           // stakes, ledger weights and the peers' gates follow the tables
     CUDA_TRY(n, cudaStreamSynchronize(n->stream));
     return launch_status(n, "import_table");
 }
@@ -565,6 +570,14 @@ wwws_status wwws_set_option(wwws_network* n, wwws_option option, int64_t value)
     case WWWS_OPT_REQUEST_KERNEL:
         if (value < 0 || value > 2) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_REQUEST_KERNEL takes 0 (by size), 1 (warp) or 2 (thread)");
         n->request_kernel = int(value);
+        return WWWS_OK;
+    case WWWS_OPT_STEP_KERNEL:
+        if (value < 0 || value > 4) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_STEP_KERNEL takes 0 (by size), 1 (8 lanes), 2 (4 lanes), 3 (thread) or 4 (streaming)");
+        n->step_kernel = int(value);
+        return WWWS_OK;
+    case WWWS_OPT_STREAM_RUN:
+        if (value < 0 || value > 65536 || value % 32) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_STREAM_RUN takes 0 (by size) or a multiple of 32 up to 65536");
+        n->stream_run = uint32_t(value);
         return WWWS_OK;
     default:
         return fail(n, WWWS_ERR_ARG, "unknown option");

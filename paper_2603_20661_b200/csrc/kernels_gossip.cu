@@ -16,8 +16,8 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
     bool on = n.online[x] != 0;
     if (n.p_leave | n.p_join) {
         const uint32_t u = ppm(draw(n, i, round, rg, kChurn).w[0]);
-        if (on) { if (u < n.p_leave) { on = false; n.backlog[x] = 0; n.online[x] = 0; } }
-        else if (u < n.p_join) { on = true; n.online[x] = 1; }
+        if (on) { if (u < n.p_leave) { on = false; n.backlog[x] = 0; n.online[x] = 0; refresh_gate(n, x, false, n.cap_eff[x], 0, n.credit[x]); } }
+        else if (u < n.p_join) { on = true; n.online[x] = 1; refresh_gate(n, x, true, n.cap_eff[x], n.backlog[x], n.credit[x]); }
     }
     int32_t part[4] = { -1, -1, -1, -1 };
     uint64_t self = 0;

@@ -38,7 +38,7 @@ __device__ __forceinline__ float score_lanes(const Net& n, Lanes<L>& w, uint32_t
     constexpr int CP = Lanes<L>::CP;
     const uint32_t c0 = w.sub * CP;
     const uint64_t* win = n.view + (size_t(r) * n.N + o) * n.ld + kWin * blk + c0;
-    const float* wled = n.w_led + size_t(r) * n.N;
+    const float* wled = n.w_led + size_t(r) * n.ld;
     uint64_t e[CP];
 #pragma unroll
     for (int j = 0; j < CP; j += 4) {
@@ -197,7 +197,7 @@ __global__ void __launch_bounds__(128) k_step_lanes(Net n, uint64_t first, uint3
                 }
             }
             if (a >= 0) {
-                if (n.score_a) candidate_weight(n, o, uint32_t(a), n.view[(pbase + o) * n.ld + a], n.w_led[pbase + a], sa);
+                if (n.score_a) candidate_weight(n, o, uint32_t(a), n.view[(pbase + o) * n.ld + a], n.w_led[size_t(r) * n.ld + a], sa);
                 if (duel) {
                     oc = 4;
                     if (found >= 0 && nj > 0) {

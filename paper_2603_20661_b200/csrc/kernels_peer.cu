@@ -31,8 +31,9 @@ __global__ void k_peer_init(Net n, const int64_t* __restrict__ credit0, const ui
     n.wins[x] = 0; n.duels[x] = 0; n.served[x] = 0; n.served_local[x] = 0;
     n.d_credit[x] = 0; n.d_wins[x] = 0; n.d_duels[x] = 0; n.d_backlog[x] = 0;
     n.blk_spent[x] = 0; n.d_spent[x] = 0;
-    n.w_led[x] = ledger_weight(n, st, 0, 0);
+    n.w_led[size_t(r) * n.ld + j] = ledger_weight(n, st, 0, 0);
     n.self_entry[x] = 0;
+    refresh_gate(n, x, online0[x] != 0, n.cap_eff[x], 0, c);
 }
 
 // V[i][j] = entry of j at a version 0..init_stale_max old (own entry current).
@@ -59,12 +60,16 @@ __global__ void k_advance(Net n, uint32_t dt_ms, uint32_t now_ms)
     if (j >= n.N) return;
     const size_t x = size_t(r) * n.N + j;
     const uint32_t cap = n.cap_eff[x];
-    if (n.online[x]) {
+    const bool on = n.online[x] != 0;
+    int64_t b = n.backlog[x];
+    if (on) {
         const int64_t done = int64_t(uint64_t(cap) * dt_ms / 1000u);
-        const int64_t b = n.backlog[x];
-        n.backlog[x] = b > done ? b - done : 0;
+        b = b > done ? b - done : 0;
+        n.backlog[x] = b;
     }
-    n.cap_eff[x] = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, now_ms);
+    const uint32_t cap_now = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, now_ms);
+    n.cap_eff[x] = cap_now;
+    refresh_gate(n, x, on, cap_now, b, n.credit[x]);
 }
 
 // Commit of replica r's block, run by the last block of k_fold to finish that replica: total
@@ -102,7 +107,9 @@ __global__ void k_fold(Net n, int finalize_requested)
     if (j < n.N) {
         const size_t x = size_t(r) * n.N + j;
         const long long db = n.d_backlog[x];
-        if (db) { n.backlog[x] += db; n.d_backlog[x] = 0; }
+        const int64_t queued = n.backlog[x] + db;
+        if (db) { n.backlog[x] = queued; n.d_backlog[x] = 0; }
+        int64_t credit_now = n.credit[x];
         if (n.flags & 16u) {
             n.in_deg[x] = 0;                         // per-peer item counts of the batch's queueing pass
             n.blk_spent[x] = finalize ? 0 : n.blk_spent[x] + n.d_spent[x];
@@ -115,9 +122,11 @@ __global__ void k_fold(Net n, int finalize_requested)
             n.d_credit[x] = 0; n.d_wins[x] = 0; n.d_duels[x] = 0;
             const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
             n.stake[x] = st;
-            n.w_led[x] = ledger_weight(n, st, w, d);
+            n.w_led[size_t(r) * n.ld + j] = ledger_weight(n, st, w, d);
             csum = c;
+            credit_now = c;
         }
+        if (db || finalize) refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], queued, credit_now);
     }
     if (finalize) {
         for (int o = 16; o; o >>= 1) csum += __shfl_down_sync(0xffffffffu, csum, o);
@@ -152,7 +161,8 @@ __global__ void k_rederive(Net n)
     const int64_t c = n.credit[x];
     const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
     n.stake[x] = st;
-    n.w_led[x] = ledger_weight(n, st, n.wins[x], n.duels[x]);
+    n.w_led[size_t(r) * n.ld + j] = ledger_weight(n, st, n.wins[x], n.duels[x]);
+    refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], n.backlog[x], c);
 }
 
 // credit_total per replica = sum of finalized and pending credit.

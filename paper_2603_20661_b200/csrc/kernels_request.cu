@@ -22,7 +22,7 @@ __device__ __forceinline__ void score_lane(const Net& n, Window& w, uint32_t lan
 {
     const uint32_t id = kWin * w.blk + lane;
     const uint64_t e = n.view[(size_t(w.r) * n.N + w.o) * n.ld + id];     // id < ld always: coalesced 256 B per warp
-    const float wl = id < n.N ? n.w_led[size_t(w.r) * n.N + id] : 0.0f;
+    const float wl = n.w_led[size_t(w.r) * n.ld + id];                   // padding columns hold 0
     w.W = candidate_weight(n, w.o, id, e, wl, w.score);
 }
 

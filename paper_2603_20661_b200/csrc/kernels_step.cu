@@ -96,7 +96,7 @@ __device__ __forceinline__ float score_window(const Net& n, StepShared<BT>& sh, 
                                               uint32_t keep, Draws& d)
 {
     const uint64_t* win = n.view + (size_t(r) * n.N + o) * n.ld + kWin * blk;
-    const float* wled = n.w_led + size_t(r) * n.N;
+    const float* wled = n.w_led + size_t(r) * n.ld;
     float ssum = 0.0f;
 #pragma unroll kScoreUnroll
     for (int g = 0; g < 4; ++g) {
@@ -238,7 +238,7 @@ __global__ void __launch_bounds__(BT, BT == 128 ? kStepBlocksPerSM : 1) k_step_f
                     if (found >= 0) {
                         a = found;
                         duel = duel_if_found;
-                        if (n.score_a) candidate_weight(n, o, uint32_t(a), n.view[(pbase + o) * n.ld + a], n.w_led[pbase + a], sa);
+                        if (n.score_a) candidate_weight(n, o, uint32_t(a), n.view[(pbase + o) * n.ld + a], n.w_led[size_t(r) * n.ld + a], sa);
                     } else a = local_code == -4 ? -4 : -2;
                 }
                 n.exec_a[x] = a;
@@ -302,10 +302,16 @@ static void launch_by_size(const Net& n, uint64_t first, uint32_t count, const L
         k_step_fused<32, MODE><<<dim3((count + 31) / 32, n.Rp), 32, 0, c.stream>>>(n, first, count);
 }
 
-void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
+void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c, int step_kernel, uint32_t stream_run)
 {
-    // launches that leave most of the GPU empty share a request among several lanes
-    if (const int lanes = step_lanes_for(uint64_t(count) * n.Rp)) { launch_step_lanes(n, first, count, lanes, c); return; }
+    if (step_kernel == 0) {
+        // launches that leave most of the GPU empty share a request among several lanes; the others
+        // are taken through the protocol phase by phase, with full warps
+        const int lanes = step_lanes_for(uint64_t(count) * n.Rp);
+        step_kernel = lanes == 8 ? 1 : lanes == 4 ? 2 : 4;
+    }
+    if (step_kernel == 1 || step_kernel == 2) { launch_step_lanes(n, first, count, step_kernel == 1 ? 8 : 4, c); return; }
+    if (step_kernel == 4) { launch_step_stream(n, first, count, stream_run, c); return; }
     Timed t(c, kStepFused);
     launch_by_size<kModeFused>(n, first, count, c);
 }

@@ -148,8 +148,51 @@ __device__ __forceinline__ void fifo_emit(const Net& n, uint32_t r, uint32_t bid
     if (peer >= 0) atomicAdd(&n.in_deg[size_t(r) * n.N + peer], 1u);
 }
 
+// S3 of a decided duel (outcome 1..3): the challenger's execution and payment, the judges' work,
+// the reputation counters and the redistribution of the penalty.  Returns what the origin pays on
+// top of the primary execution (R, for the challenger's run); the caller books it on the origin.
+template <class Acc>
+__device__ __forceinline__ long long settle_duel(const Net& n, uint32_t r, uint32_t q, uint32_t o, uint32_t li, uint32_t lo,
+                                                 int a, int b, const int (&jd)[4], uint32_t oc, Acc& s)
+{
+    const size_t base = size_t(r) * n.N;
+    const uint64_t key = chain_key(n, r);
+    const uint64_t work = uint64_t(li) + lo;
+    s.digest += record_hash(key, q, opPayChallenger, o, -n.R) + record_hash(key, q, opEarnChallenger, uint32_t(b), n.R);
+    add64(&n.d_credit[base + b], n.R);
+    add64(&n.d_backlog[base + b], (long long)work);
+    atomicAdd(&n.served[base + b], 1ull);
+    atomicAdd(&n.d_duels[base + a], 1u);
+    atomicAdd(&n.d_duels[base + b], 1u);
+    int nj = 0;
+#pragma unroll
+    for (int l = 0; l < 4; ++l)
+        if (jd[l] >= 0) { add64(&n.d_backlog[base + jd[l]], (long long)(uint64_t(li) + 2ull * lo)); ++nj; }
+    s.add(sJudgeEvals, uint32_t(nj));
+    if (oc == 3) s.add(sDraw);
+    else {
+        const int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
+        const long long pot = n.P - n.R_add, share = n.judge_share[nj - 1];
+        const long long prize = n.R_add + (pot - share * nj);
+        s.digest += record_hash(key, q, opPenalty, uint32_t(lose), -n.P) + record_hash(key, q, opReward, uint32_t(win), prize);
+        add64(&n.d_credit[base + lose], -n.P);
+        add64(&n.d_credit[base + win], prize);
+        atomicAdd(&n.d_wins[base + win], 1u);
+#pragma unroll
+        for (int l = 0; l < 4; ++l)
+            if (jd[l] >= 0) {
+                s.digest += record_hash(key, q, opJudge + l, uint32_t(jd[l]), share);
+                add64(&n.d_credit[base + jd[l]], share);
+            }
+    }
+    return n.R;
+}
+
+// Settlement of one request.  `duel_booked`: the caller has already run settle_duel for this request
+// (and booked its extra payment on the origin); everything else is still done here.
+template <class Acc>
 __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q, uint32_t bidx, uint32_t o, uint32_t li, uint32_t lo,
-                                           int a, int b, const int (&jd)[4], uint32_t oc, bool near, SettleAcc& s)
+                                           int a, int b, const int (&jd)[4], uint32_t oc, bool near, Acc& s, bool duel_booked = false)
 {
     if (n.flags & 16u) {
         const bool served = a != -3 && a != -4, duel = a >= 0 && oc >= 1 && oc <= 3;
@@ -185,36 +228,7 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
         ex = uint32_t(a);
         if (oc != 0) s.add(sDuel);
         if (oc == 4) s.add(sDuelCancelled);
-        if (oc >= 1 && oc <= 3) {
-            pay += n.R;
-            s.digest += record_hash(key, q, opPayChallenger, o, -n.R) + record_hash(key, q, opEarnChallenger, uint32_t(b), n.R);
-            add64(&n.d_credit[base + b], n.R);
-            add64(&n.d_backlog[base + b], (long long)work);
-            atomicAdd(&n.served[base + b], 1ull);
-            atomicAdd(&n.d_duels[base + a], 1u);
-            atomicAdd(&n.d_duels[base + b], 1u);
-            int nj = 0;
-#pragma unroll
-            for (int l = 0; l < 4; ++l)
-                if (jd[l] >= 0) { add64(&n.d_backlog[base + jd[l]], (long long)(uint64_t(li) + 2ull * lo)); ++nj; }
-            s.add(sJudgeEvals, uint32_t(nj));
-            if (oc == 3) s.add(sDraw);
-            else {
-                const int win = oc == 1 ? a : b, lose = oc == 1 ? b : a;
-                const long long pot = n.P - n.R_add, share = n.judge_share[nj - 1];
-                const long long prize = n.R_add + (pot - share * nj);
-                s.digest += record_hash(key, q, opPenalty, uint32_t(lose), -n.P) + record_hash(key, q, opReward, uint32_t(win), prize);
-                add64(&n.d_credit[base + lose], -n.P);
-                add64(&n.d_credit[base + win], prize);
-                atomicAdd(&n.d_wins[base + win], 1u);
-#pragma unroll
-                for (int l = 0; l < 4; ++l)
-                    if (jd[l] >= 0) {
-                        s.digest += record_hash(key, q, opJudge + l, uint32_t(jd[l]), share);
-                        add64(&n.d_credit[base + jd[l]], share);
-                    }
-            }
-        }
+        if (oc >= 1 && oc <= 3 && !duel_booked) pay += settle_duel(n, r, q, o, li, lo, a, b, jd, oc, s);
         add64(&n.d_credit[base + o], -pay);
     }
     if (n.flags & 16u) return;                       // latency and SLO are counted by k_fifo_latency

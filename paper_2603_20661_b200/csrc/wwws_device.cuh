@@ -46,8 +46,12 @@ struct Net {
     unsigned long long* served; unsigned long long* served_local;
     // pending block and pending queue growth
     long long* d_credit; uint32_t* d_wins; uint32_t* d_duels; long long* d_backlog;
-    // derived: (float)stake * smoothed win rate, refreshed whenever the ledger is finalized
+    // derived: (float)stake * smoothed win rate, refreshed whenever the ledger is finalized; [Rp][ld], padding 0,
+    // so that a candidate window's 32 weights are one aligned 128-byte segment
     float* w_led;
+    // derived: what a probe and an origin decision need from a peer's true state and policy, in one word each
+    // (see peer_gate); refreshed by every kernel that changes online, cap_eff, backlog or the finalized credit
+    uint64_t* gate;
     // gossip scratch: this round's self entries and chosen partners
     uint64_t* self_entry; int32_t* partner;     // partner is [Rp][N][4]
     // reverse lists of the pairwise exchange: in-degree, list offset, fill cursor, puller ids [Rp][4N]
@@ -111,6 +115,24 @@ __device__ __forceinline__ bool util_at_least(uint32_t cap_eff, int64_t backlog,
     uint64_t denom = uint64_t(cap_eff) * util_window_ms / 1000u;
     if (denom < 1) denom = 1;
     return uint64_t(backlog) * 1000ull >= uint64_t(thr) * denom;
+}
+
+// A peer's "gate": everything a probe of the peer (low word) and a dispatch decision at the peer as
+// origin (high word) read from its true state and policy, evaluated once per state change instead
+// of once per request.
+//   low  word: accept frequency in ppm if the peer would accept delegated work now (online, has
+//              capacity, utilisation below its accept threshold), else 0: a probe is  ppm(u) < low
+//   high word: bits 0..19 offload frequency in ppm if the peer, as origin, may offload now
+//              (utilisation at or above its threshold and it can afford R), else 0;
+//              bit 20 online; bit 21 no capacity
+constexpr uint32_t kGateOnline = 1u << 20, kGateNoCap = 1u << 21, kGateFreq = (1u << 20) - 1u;
+__device__ __forceinline__ void refresh_gate(const Net& n, size_t x, bool on, uint32_t cap, int64_t backlog, int64_t credit)
+{
+    const bool accepts = on && cap != 0 && !util_at_least(cap, backlog, n.util_window_ms, n.accept_util_pm[x]);
+    const bool offloads = util_at_least(cap, backlog, n.util_window_ms, n.offload_util_pm[x]) && credit >= n.R;
+    const uint32_t lo = accepts ? n.accept_ppm[x] : 0u;
+    const uint32_t hi = (offloads ? n.offload_ppm[x] : 0u) | (on ? kGateOnline : 0u) | (cap == 0 ? kGateNoCap : 0u);
+    n.gate[x] = uint64_t(hi) << 32 | lo;
 }
 
 __device__ __forceinline__ uint32_t cap_eff_at(const Net& n, uint32_t cap_true, bool prio, uint32_t j, uint32_t rg,

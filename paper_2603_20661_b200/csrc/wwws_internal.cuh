@@ -49,7 +49,10 @@ void launch_fifo(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& 
 void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_duel(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
 void launch_settle(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
-void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);
+// step_kernel: 0 chosen by launch size, 1 eight lanes per request, 2 four lanes, 3 one thread per request,
+// 4 streaming phases; stream_run: requests per warp of the streaming kernel, 0 = by launch size
+void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c, int step_kernel = 0, uint32_t stream_run = 0);
+void launch_step_stream(const Net& n, uint64_t first, uint32_t count, uint32_t per_warp, const LaunchCtx& c);
 int step_lanes_for(uint64_t total_requests);
 void launch_step_lanes(const Net& n, uint64_t first, uint32_t count, int lanes, const LaunchCtx& c);
 void launch_dispatch_threads(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c);

@@ -108,22 +108,67 @@ def test_fused_step_matches_oracle(name, kw, steps):
     assert_same_state(g, o, "fused end", upto=wl.n_requests)
 
 
-@pytest.mark.parametrize("batch,flags", [(250, 3), (1500, 3), (5000, 3), (10000, 3), (250, 7), (1500, 7), (1500, 19)],
-                         ids=["8_lanes", "4_lanes", "thread_blocks_of_32", "thread_blocks_of_128", "8_lanes_greedy", "4_lanes_greedy",
-                              "4_lanes_fifo"])
-def test_fused_step_at_every_launch_size_matches_oracle(batch, flags):
-    """The fused step picks its kernel by launch size (8 or 4 lanes per request, one thread per
-    request in blocks of 32 or 128): 8 replicas x batch = 2,000 / 12,000 / 40,000 / 80,000 requests."""
+STEP_KERNELS = {"8_lanes": 1, "4_lanes": 2, "thread": 3, "stream": 4}
+
+
+@pytest.mark.parametrize("batch,flags,kernel,run", [
+    (250, 3, "8_lanes", 0), (1500, 3, "4_lanes", 0), (5000, 3, "thread", 0), (10000, 3, "thread", 0),
+    (250, 7, "8_lanes", 0), (1500, 7, "4_lanes", 0), (1500, 19, "4_lanes", 0), (5000, 7, "thread", 0),
+    (250, 3, "stream", 32), (1500, 3, "stream", 64), (5000, 3, "stream", 0), (5000, 3, "stream", 512), (10000, 3, "stream", 96),
+    (10000, 3, "stream", 0), (1500, 7, "stream", 64), (5000, 19, "stream", 160), (5000, 0, "stream", 0), (1500, 35, "stream", 2048),
+    (5000, 3, None, 0), (10000, 3, None, 0)],
+    ids=lambda v: str(v))
+def test_fused_step_with_every_kernel_matches_oracle(batch, flags, kernel, run):
+    """The fused step has four implementations with identical results (8 or 4 lanes per request,
+    one thread per request, streaming phases with runs of `run` requests per warp); each is forced
+    on here, and left to the launch size in the last two cases: 8 replicas x batch = 2,000 /
+    12,000 / 40,000 / 80,000 requests per launch."""
     wl = synth.make_workload("zipf1k", n_replicas=8, n_requests=2 * batch, n_peers=300)
     wl.batch = batch
     wl.settings.flags = flags
     wl.settings.p_duel_ppm = 150_000
     g, o = _pair(wl)
+    if kernel:
+        g.set_option(1, STEP_KERNELS[kernel])
+        g.set_option(2, run)
     for s in range(2):
         g.step(s * batch, batch, wl.step_now_ms(s), s == 0, s == 1)
         o.run_step(s * batch, batch, wl.step_now_ms(s), s == 0, s == 1)
         assert_same_state(g, o, f"batch {batch} step {s}", upto=(s + 1) * batch, views=s == 0)
     assert o.stats_dict()["n_duel"] > 0.05 * o.stats_dict()["n_delegated"] > 0
+
+
+@pytest.mark.parametrize("case", ["all_duels_four_judges", "one_probe", "nobody_accepts", "all_local", "ragged_window", "no_scores"])
+def test_streaming_kernel_corner_cases_match_oracle(case):
+    """The streaming kernel where its queues are stressed: every delegated request a duel with four
+    judges (the draw queue recirculates), a probe budget of one, nobody accepting (all fall back),
+    nobody offloading (everything goes straight to the finish queue), a last candidate block of 12."""
+    kw = dict(n_replicas=3, n_requests=3000, n_peers=300)
+    if case == "ragged_window":
+        kw["n_peers"] = 44
+    wl = synth.make_workload("zipf1k", **kw)
+    wl.batch = 1500
+    st = wl.settings
+    if case == "all_duels_four_judges":
+        st.p_duel_ppm, st.n_judges, st.p_noise_ppm = 1_000_000, 4, 200_000
+    elif case == "one_probe":
+        st.max_probes, st.p_duel_ppm = 1, 400_000
+    elif case == "nobody_accepts":
+        wl.peers["accept_ppm"][:] = 0
+    elif case == "all_local":
+        wl.peers["offload_ppm"][:] = 0
+    elif case == "ragged_window":
+        st.rank_cdf = None
+        st.p_duel_ppm = 500_000
+    g, o = _pair(wl)
+    if case == "no_scores":
+        g.bind_requests(wl.requests, scores=False)
+    g.set_option(1, 4)
+    for s in range(2):
+        g.set_option(2, (96, 0)[s])
+        g.step(s * 1500, 1500, wl.step_now_ms(s), s == 0, True)
+        o.run_step(s * 1500, 1500, wl.step_now_ms(s), s == 0, True)
+        assert_same_state(g, o, f"{case} step {s}", upto=(s + 1) * 1500, views=s == 0, scores=case != "no_scores")
 
 
 @pytest.mark.parametrize("pinned", [True, False], ids=["mapped_host_buffers", "pageable_host_buffers"])
@@ -285,6 +330,9 @@ def test_random_configurations_match_oracle(seed):
     rq["len_out"] = rng.integers(1, 8193, (Rp, Q)).astype(np.uint16)
     g = Network(st, pa, B); g.bind_requests(rq)
     g.set_option(0, 1 + seed % 2)                # six-call path: warp-per-request / thread-per-request kernels in turn
+    g.set_option(1, (0, 3, 4)[seed % 3])         # fused step: by launch size / one thread per request / streaming phases
+    if seed % 3 == 2:
+        g.set_option(2, int(rng.choice([0, 32, 64, 224])))
     o = Oracle(st, pa); o.bind_requests(rq)
     assert_same_state(g, o, f"seed {seed} create")
     first, step = 0, 0
