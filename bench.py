@@ -7,13 +7,17 @@ A step is one pass of the whole path over one batch: advance -> gossip (on the s
 cadence selects) -> dispatch -> duel-and-judge -> settle.  Metric: simulated requests
 dispatched and settled per second.  One JSON line is printed by rank 0.
 
-Multi-GPU (`torchrun`, one process per GPU): replicas are independent, so every rank runs its
-own set of replicas (weak scaling, no data-path collective); timing is the max over ranks.
+Multi-GPU: replicas are independent, so every rank runs its own set of replicas (weak
+scaling, no data-path collective; only counters and the max-over-ranks time are reduced).
+`--gpus N` with N > 1 starts N ranks itself (one process per GPU through torch.distributed.run)
+unless it already runs under such a launcher (WORLD_SIZE set).
 `--impl reference` times the CPU oracle, as it stands, on a bounded sample of the workload.
 """
 from __future__ import annotations
 
 import argparse
+import glob
+import hashlib
 import json
 import os
 import statistics
@@ -29,12 +33,9 @@ sys.path.insert(0, ROOT)
 METRIC = "simulated requests dispatched+settled per second"
 UNIT = "requests/s"
 DEFAULT_WORKLOAD = "adversarial16k"          # the largest single-GPU configuration
-
-
-# DRAM traffic (read + write) of one k_gossip_merge pass over one replica, from the ncu capture
-# summarised in profiles/k_gossip_merge_adversarial16k_1replica.md; a launch over Rp replicas is
-# Rp such passes back to back (replica-major grid), so traffic scales with the replica count.
-NCU_MERGE_TRAFFIC = {"n_peers": 16384, "fanout_k": 4, "flags": 3, "bytes_per_replica": 2.1897e9 + 2.1133e9}
+EXTRA_LEGS = ("zipf1k", "churn4k")           # also timed, compactly, by the default run
+TARGET_FRAC = 0.6                            # the stated goal for dispatch+settle: 60 % of HBM bandwidth
+N_SM, ISSUE_PER_SM = 148, 4                  # warp instructions an SM can issue per cycle: one per scheduler
 
 
 def measured_peaks():
@@ -43,6 +44,41 @@ def measured_peaks():
         with open(p) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def read_counter_files():
+    """Counters taken from ncu captures: `profiles/*_counters.txt`, one capture per file, `key: value`
+    lines (kernel, workload, commit, source file and its sha256 at the time of the capture, figures)."""
+    out = []
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*_counters.txt"))):
+        rec = {"file": os.path.relpath(path, ROOT)}
+        with open(path) as f:
+            for ln in f:
+                if ln.startswith("#") or ":" not in ln:
+                    continue
+                k, v = ln.split(":", 1)
+                rec[k.strip()] = v.strip()
+        out.append(rec)
+    return out
+
+
+def source_unchanged(rec):
+    """True if the kernel's source file still has the digest recorded with the capture."""
+    src = rec.get("source")
+    if not src or "source_sha256" not in rec:
+        return False
+    try:
+        with open(os.path.join(ROOT, src), "rb") as f:
+            return hashlib.sha256(f.read()).hexdigest() == rec["source_sha256"]
+    except OSError:
+        return False
+
+
+def find_counters(kernel, **match):
+    for rec in read_counter_files():
+        if rec.get("kernel") == kernel and all(str(rec.get(k)) == str(v) for k, v in match.items()):
+            return rec
+    return None
 
 
 class ClockSampler:
@@ -60,6 +96,8 @@ class ClockSampler:
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
+        time.sleep(0.5)                                # nvidia-smi needs a moment before its first sample
+        return self
 
     def stop(self):
         if not self.proc:
@@ -83,8 +121,8 @@ class ClockSampler:
             for nm, v in zip(names, f[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def step_args(wl, s, phase=0):
@@ -101,10 +139,10 @@ def step_args(wl, s, phase=0):
 
 
 def algorithmic_bytes(wl, stats_delta):
-    """Bytes the method must move (stated in the design notes):
-    gossip round: 2 * 8 * N^2 per replica (every view entry read once and written once; the
-    k+1 readers of a row share it through L2 because the merge walks the matrix by column panels);
-    request path: 8 B record + 26 B result, plus a 256 B view window per request that offloads."""
+    """Bytes the method must move.
+    Gossip round: 2 * 8 * N^2 per replica (every view entry read once and written once; the k+1
+    readers of a row share it through L2 because the merge walks the matrix by column panels).
+    Request path: 8 B record + 26 B result, plus a 256 B view window per request that offloads."""
     st = wl.settings
     gossip_round = 2 * 8 * st.n_peers ** 2 * st.n_replicas
     offloaded = stats_delta["n_delegated"] + stats_delta["n_fallback_local"] + stats_delta["n_failed"]
@@ -112,91 +150,97 @@ def algorithmic_bytes(wl, stats_delta):
     return gossip_round, req
 
 
-def run_gpu(args):
-    import torch
-    import torch.distributed as dist
-    from paper_2603_20661_b200 import synth
-    from paper_2603_20661_b200.binding import Network, STAT_NAMES
+REQUEST_KERNELS = ("k_advance", "k_step_fused", "k_fold", "k_fifo")
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    torch.cuda.set_device(local)
-    dev = torch.device(f"cuda:{local}")
 
-    from paper_2603_20661_b200.sharding import max_over_ranks, replica_shard, sum_counters
-    wl0 = synth.make_workload(args.workload, seed=args.seed, n_replicas=args.replicas)
-    Rp = wl0.settings.n_replicas
-    # weak scaling: every rank runs the configuration's full replica count, on its own replica indices
-    off, _ = replica_shard(world * Rp, world, rank)
-    wl = synth.make_workload(args.workload, seed=args.seed, replica_offset=off, n_replicas=args.replicas)
-    if args.batch:
-        wl.batch = args.batch
-    wl.settings.flags |= (8 if args.push_pull else 0) | (4 if args.greedy else 0)
-    st = wl.settings
-    net = Network(st, wl.peers, wl.batch, device=dev)
-    net.bind_requests(wl.requests, scores=False)
+class Leg:
+    """One workload on this rank's GPU: the network, its step counter and the timed regions."""
 
-    def barrier():
-        if world > 1:
+    def __init__(self, args, name, dev, world, rank, batch=None):
+        import torch
+        from paper_2603_20661_b200 import synth
+        from paper_2603_20661_b200.binding import Network
+        from paper_2603_20661_b200.sharding import replica_shard
+        self.torch, self.dev, self.world, self.rank, self.name = torch, dev, world, rank, name
+        wl0 = synth.make_workload(name, seed=args.seed, n_replicas=args.replicas)
+        self.Rp = wl0.settings.n_replicas
+        # weak scaling: every rank runs the configuration's full replica count, on its own replica indices
+        off, _ = replica_shard(world * self.Rp, world, rank)
+        self.wl = synth.make_workload(name, seed=args.seed, replica_offset=off, n_replicas=args.replicas)
+        if batch:
+            self.wl.batch = batch
+        self.wl.settings.flags |= (8 if args.push_pull else 0) | (4 if args.greedy else 0)
+        self.net = Network(self.wl.settings, self.wl.peers, self.wl.batch, device=dev)
+        self.net.bind_requests(self.wl.requests, scores=False)
+        if args.step_kernel:
+            self.net.set_option(1, args.step_kernel)
+        if args.stream_run:
+            self.net.set_option(2, args.stream_run)
+        self.W, self.s = args.warmup, 0
+        for _ in range(self.W):
+            f, c, now, g = step_args(self.wl, self.s, self.W)
+            self.net.step(f, c, now, g or self.s == 0); self.s += 1     # a gossip round in the warm-up whatever the phase
+        self.align()
+
+    def close(self):
+        self.net.close()
+        self.net = None
+        self.torch.cuda.empty_cache()
+
+    def barrier(self):
+        if self.world > 1:
+            import torch.distributed as dist
             dist.barrier()
-        torch.cuda.synchronize(dev)
+        self.torch.cuda.synchronize(self.dev)
 
-    reduce_max, reduce_sum_vec = max_over_ranks, sum_counters
+    def totals(self):
+        from paper_2603_20661_b200.binding import STAT_NAMES
+        return dict(zip(STAT_NAMES, (int(v) for v in self.net.stats()[-1])))
 
-    W, K = args.warmup, args.steps
-    s = 0
-    for _ in range(W):
-        f, c, now, g = step_args(wl, s, W)
-        net.step(f, c, now, g or s == 0); s += 1        # a gossip round in the warm-up whatever the phase
-    stats0 = net.stats()[-1].copy()
-    launches0 = net.kernel_launches()
+    def align(self, call=None):
+        """Run untimed steps until the next step is a gossip step, as the first timed region starts."""
+        call = call or self.net.step
+        while (self.s - self.W) % self.wl.gossip_every:
+            call(*step_args(self.wl, self.s, self.W)); self.s += 1
 
-    # ---- timed region A: device-resident inputs --------------------------------------------
-    sampler = ClockSampler(local) if rank == 0 else None
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if sampler:
-        sampler.start()
-        time.sleep(0.5)                                # nvidia-smi needs a moment before its first sample
-    barrier()
-    ev0.record()
-    for _ in range(K):
-        net.step(*step_args(wl, s, W)); s += 1
-    ev1.record()
-    barrier()
-    ms = reduce_max(ev0.elapsed_time(ev1))
-    launches = net.kernel_launches() - launches0
-    stats1 = net.stats()[-1].copy()
-    delta = {k: int(b) - int(a) for k, a, b in zip(STAT_NAMES, stats0, stats1)}
-    total_requests = int(reduce_sum_vec(np.array([delta["n_requests"]], np.uint64))[0])
-    value = total_requests / (ms * 1e-3)
+    def timed(self, K, call=None, repeats=1):
+        """`repeats` back-to-back regions of K steps, each bracketed by CUDA events on the launching
+        stream, barrier + synchronize on both sides of the whole; returns the per-region times (ms,
+        max over ranks) and the counter deltas of all regions together."""
+        from paper_2603_20661_b200.sharding import max_over_ranks
+        torch = self.torch
+        call = call or self.net.step
+        before = self.totals()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+        self.barrier()
+        ev[0].record()
+        for i in range(repeats):
+            for _ in range(K):
+                call(*step_args(self.wl, self.s, self.W)); self.s += 1
+            ev[i + 1].record()
+        self.barrier()
+        ms = [max_over_ranks(ev[i].elapsed_time(ev[i + 1])) for i in range(repeats)]
+        after = self.totals()
+        return ms, {k: after[k] - before[k] for k in after}
 
-    # a second, identical timed region: reported beside the first one so that a disturbed run shows
-    barrier()
-    ev0.record()
-    for _ in range(K):
-        net.step(*step_args(wl, s, W)); s += 1
-    ev1.record()
-    barrier()
-    ms_repeat = reduce_max(ev0.elapsed_time(ev1))
+    def profiled(self, K):
+        """K steps with per-kernel events: {kernel: (summed ms, launches)} and the counter deltas."""
+        before = self.totals()
+        self.net.profile(True)
+        for _ in range(K):
+            self.net.step(*step_args(self.wl, self.s, self.W)); self.s += 1
+        prof = self.net.profile_read()
+        self.net.profile(False)
+        after = self.totals()
+        return prof, {k: after[k] - before[k] for k in after}
 
-    # ---- region B: same K steps with per-kernel events (roofline of the dominant kernel) ---
-    net.profile(True)
-    stats_b0 = net.stats()[-1].copy()
-    for _ in range(K):
-        net.step(*step_args(wl, s, W)); s += 1
-    prof = net.profile_read()
-    net.profile(False)
-    clocks = sampler.stop() if sampler else None     # sampled over region A and its instrumented repeat
-    stats_b1 = net.stats()[-1].copy()
-    delta_b = {k: int(b) - int(a) for k, a, b in zip(STAT_NAMES, stats_b0, stats_b1)}
+
+def rooflines(leg, prof, delta_b, sm_mhz):
+    """HBM roofline of the gossip merge and of the request kernel, and the issue-slot roofline of
+    the request kernel (warp instructions per request from the ncu capture on record)."""
+    st, wl = leg.wl.settings, leg.wl
     peak, peak_kind = measured_peaks()
     g_bytes, req_bytes = algorithmic_bytes(wl, delta_b)
-    total_ms = sum(v[0] for v in prof.values())
-    dom = max(prof, key=lambda k: prof[k][0])
-    kernels = {k: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_ms} for k, v in prof.items()}
 
     def roof(kernel, bytes_per_launch):
         if kernel not in prof:
@@ -204,43 +248,137 @@ def run_gpu(args):
         t = prof[kernel][0] / prof[kernel][1] * 1e-3
         ach = bytes_per_launch / t / 1e9
         return {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "peak_source": peak_kind, "traffic": None, "bytes_per_launch": bytes_per_launch,
-                "ms_per_launch": t * 1e3}
+                "peak_source": peak_kind, "traffic": None, "bytes_per_launch": bytes_per_launch, "ms_per_launch": t * 1e3}
 
-    roof_merge = roof("k_gossip_merge", g_bytes)
-    if roof_merge and (st.n_peers, st.fanout_k, st.flags) == tuple(NCU_MERGE_TRAFFIC[k] for k in ("n_peers", "fanout_k", "flags")):
-        roof_merge["traffic"] = NCU_MERGE_TRAFFIC["bytes_per_replica"] * Rp
-    if roof_merge:      # context: bytes a merge without L2 reuse would move (k+1 rows read, one written)
-        roof_merge["bytes_per_launch_without_reuse"] = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
-    roof_req = roof("k_step_fused", req_bytes / max(1, prof.get("k_step_fused", (0, 1))[1]))
+    merge = roof("k_gossip_merge", g_bytes)
+    if merge:
+        rec = find_counters("k_gossip_merge", n_peers=st.n_peers, fanout_k=st.fanout_k, flags=st.flags & ~4)
+        if rec and source_unchanged(rec):      # DRAM bytes of one replica's pass; a launch is Rp such passes back to back
+            merge["traffic"] = float(rec["dram_bytes_per_replica_round"]) * leg.Rp
+            merge["traffic_from_profile"] = rec["file"]
+        elif rec:
+            merge["traffic_from_profile"] = rec["file"] + " (kernel source changed since: traffic withheld)"
+        merge["bytes_per_launch_without_reuse"] = (st.fanout_k + 2) * 8 * st.n_peers ** 2 * st.n_replicas
+    launches = max(1, prof.get("k_step_fused", (0, 1))[1])
+    req = roof("k_step_fused", req_bytes / launches)
+    if req:
+        req["target_frac"] = TARGET_FRAC
+        req["target_met"] = bool(req["frac"] >= TARGET_FRAC)
+        per_launch = delta_b["n_requests"] / launches
+        rate = per_launch / (req["ms_per_launch"] * 1e-3)
+        req["requests_per_launch"] = per_launch
+        req["requests_per_s"] = rate
+        rec = find_counters("k_step_fused", workload=leg.name)
+        if rec and sm_mhz:
+            ipr = float(rec["warp_instructions_per_request"])
+            req["issue"] = {"bound": "alu", "warp_instr_per_request": ipr,
+                            "active_lanes": float(rec.get("active_lanes_per_instruction", "nan")),
+                            "issue_frac": ipr * rate / (N_SM * ISSUE_PER_SM * sm_mhz * 1e6),
+                            "peak": "148 SMs x 4 warp instructions per cycle x the SM clock sampled in this run",
+                            "sm_mhz": sm_mhz, "source": rec["file"],
+                            "source_current": source_unchanged(rec), "commit": rec.get("commit")}
+    t_req = sum(prof[k][0] for k in REQUEST_KERNELS if k in prof)
+    return merge, req, t_req
+
+
+def run_compact_leg(args, name, dev, world, rank, sampler_index):
+    """A secondary workload: value, time per step and the rooflines of its two main kernels."""
+    leg = Leg(args, name, dev, world, rank)
+    K = args.steps
+    sampler = ClockSampler(sampler_index).start() if rank == 0 else None
+    ms, delta = leg.timed(K)
+    leg.align()
+    prof, delta_b = leg.profiled(K)
+    clocks = sampler.stop() if sampler else {"sm_mhz": None}
+    merge, req, t_req = rooflines(leg, prof, delta_b, clocks.get("sm_mhz"))
+    from paper_2603_20661_b200.sharding import sum_counters
+    total = int(sum_counters(np.array([delta["n_requests"]], np.uint64))[0])
+    out = {"workload": name, "value": total / (ms[0] * 1e-3), "unit": UNIT, "ms_per_step": ms[0] / K,
+           "requests_per_step_per_gpu": leg.Rp * leg.wl.batch,
+           "gossip_merge": {k: merge[k] for k in ("frac", "ms_per_launch", "achieved")} if merge else None,
+           "request_path": ({"frac": req["frac"], "ms_per_launch": req["ms_per_launch"], "requests_per_s": req["requests_per_s"],
+                             "issue_frac": req.get("issue", {}).get("issue_frac"),
+                             "warp_instr_per_request": req.get("issue", {}).get("warp_instr_per_request")} if req else None),
+           "dispatch_duel_settle_only_ms_per_step": t_req / K, "sm_mhz": clocks.get("sm_mhz")}
+    g_a, req_a = algorithmic_bytes(leg.wl, delta)
+    out["whole_step_hbm_frac"] = (g_a * (delta["rounds"] // leg.Rp) + req_a) / (ms[0] * 1e-3) / 1e9 / measured_peaks()[0]
+    leg.close()
+    return out
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2603_20661_b200.binding import STAT_NAMES
+    from paper_2603_20661_b200.sharding import sum_counters
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE is {world}")
+    if torch.cuda.device_count() <= local:
+        raise SystemExit(f"bench.py: rank {rank} needs cuda:{local} but only {torch.cuda.device_count()} device(s) are visible")
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+
+    leg = Leg(args, args.workload, dev, world, rank, batch=args.batch)
+    wl, st, Rp, net = leg.wl, leg.wl.settings, leg.Rp, leg.net
+    K, W = args.steps, args.warmup
+    launches0 = net.kernel_launches()
+
+    # ---- region A: exactly K steps, device-resident inputs: the headline value --------------------
+    sampler = ClockSampler(local).start() if rank == 0 else None
+    ms_a, delta = leg.timed(K)
+    ms = ms_a[0]
+    launches = net.kernel_launches() - launches0
+    total_requests = int(sum_counters(np.array([delta["n_requests"]], np.uint64))[0])
+    value = total_requests / (ms * 1e-3)
+    clocks = sampler.stop() if sampler else None
+
+    # ---- sustained: the same region repeated back to back for about a second of device time (each
+    # repeat a whole number of gossip periods, so that all repeats hold the same work)
+    leg.align()
+    k_rep = K if K % wl.gossip_every == 0 else K * wl.gossip_every
+    reps = int(min(400, max(3, np.ceil(args.sustain_s * 1e3 / max(ms * k_rep / K, 1e-3)))))
+    sampler = ClockSampler(local).start() if rank == 0 else None
+    ms_rep, _ = leg.timed(k_rep, repeats=reps)
+    clocks_sustained = sampler.stop() if sampler else None
+    per_step = [m / k_rep for m in ms_rep]
+    sustained = {"repeats": len(ms_rep), "steps_per_repeat": k_rep, "device_seconds": sum(ms_rep) * 1e-3,
+                 "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
+                 "ms_per_step_max": max(per_step),
+                 "value_at_median": Rp * wl.batch * world / (statistics.median(per_step) * 1e-3),
+                 "clocks": clocks_sustained}
+
+    # ---- region B: K steps with per-kernel events (rooflines of the dominant kernel and of the request path)
+    leg.align()
+    prof, delta_b = leg.profiled(K)
+    peak, peak_kind = measured_peaks()
+    total_ms = sum(v[0] for v in prof.values())
+    dom = max(prof, key=lambda k: prof[k][0])
+    kernels = {k: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_ms} for k, v in prof.items()}
+    sm_mhz = (clocks_sustained or {}).get("sm_mhz") or (clocks or {}).get("sm_mhz")
+    roof_merge, roof_req, t_req = rooflines(leg, prof, delta_b, sm_mhz)
     roofline = roof_merge if dom == "k_gossip_merge" else roof_req
     # the whole timed region A against HBM: algorithmic bytes of its gossip rounds and requests over its duration
     g_a, req_a = algorithmic_bytes(wl, delta)
-    rounds_a = delta["rounds"] // Rp
-    step_bytes = g_a * rounds_a + req_a
+    step_bytes = g_a * (delta["rounds"] // Rp) + req_a
     whole = {"bound": "hbm", "achieved": step_bytes / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
              "frac": step_bytes / (ms * 1e-3) / 1e9 / peak, "bytes_per_step": step_bytes / K,
              "what": "all kernels of the K timed steps (gossip at its cadence + dispatch + duel + settle), algorithmic bytes"}
-    # requests/s of dispatch+duel+settle alone (advance, fused step, fold, block commit), from the same events
-    t_req = sum(prof[k][0] for k in ("k_advance", "k_step_fused", "k_fold", "k_fifo") if k in prof)
     req_only = {"value": delta_b["n_requests"] / (t_req * 1e-3), "unit": UNIT, "ms_per_step": t_req / K,
                 "kernels": "k_advance + k_step_fused + k_fold (block commit included), summed CUDA-event time"}
 
     # ---- region S: the same K steps through the six separate calls ------------------------------
-    for _ in range(min(W, 3)):                 # first use of the separate kernels loads their code: keep that untimed
-        net.run_step(*step_args(wl, s, W)); s += 1
-    while (s - W) % wl.gossip_every:
-        net.step(*step_args(wl, s, W)); s += 1
-    stats_s0 = net.stats()[-1].copy()
-    barrier()
-    ev0.record()
-    for _ in range(K):
-        net.run_step(*step_args(wl, s, W)); s += 1
-    ev1.record()
-    barrier()
-    ms_six = reduce_max(ev0.elapsed_time(ev1))
-    req_six = int(reduce_sum_vec(np.array([int(net.stats()[-1][0]) - int(stats_s0[0])], np.uint64))[0])
-    six = {"value": req_six / (ms_six * 1e-3), "unit": UNIT, "ms_per_step": ms_six / K,
+    for _ in range(3):                         # first use of the separate kernels loads their code: keep that untimed
+        net.run_step(*step_args(wl, leg.s, W)); leg.s += 1
+    leg.align()
+    ms_six, d_six = leg.timed(K, call=net.run_step)
+    req_six = int(sum_counters(np.array([d_six["n_requests"]], np.uint64))[0])
+    six = {"value": req_six / (ms_six[0] * 1e-3), "unit": UNIT, "ms_per_step": ms_six[0] / K,
            "entry": "wwws_advance_time, wwws_gossip_round, wwws_dispatch_batch, wwws_duel_judge, wwws_settle_credits"}
 
     # ---- region C: end to end through host buffers ---------------------------------------------
@@ -253,19 +391,12 @@ def run_gpu(args):
           "judges": torch.empty((Rp, Q, 4), dtype=torch.int32).pin_memory(),
           "outcome": torch.empty((Rp, Q), dtype=torch.uint8).pin_memory(),
           "flags": torch.empty((Rp, Q), dtype=torch.uint8).pin_memory()}
-    for _ in range(min(W, 3)):
-        net.step_host(io, *step_args(wl, s, W)); s += 1
-    while (s - W) % wl.gossip_every:           # start the timed steps on a gossip step, as region A did
-        net.step_host(io, *step_args(wl, s, W)); s += 1
-    stats_c0 = net.stats()[-1].copy()
-    barrier()
-    ev0.record()
-    for _ in range(K):
-        tot = net.step_host(io, *step_args(wl, s, W)); s += 1
-    ev1.record()
-    barrier()
-    ms_e2e = reduce_max(ev0.elapsed_time(ev1))
-    req_e2e = int(reduce_sum_vec(np.array([int(tot[0]) - int(stats_c0[0])], np.uint64))[0])
+    host_step = lambda *a: net.step_host(io, *a)
+    for _ in range(3):
+        host_step(*step_args(wl, leg.s, W)); leg.s += 1
+    leg.align(host_step)
+    ms_e2e, d_e2e = leg.timed(K, call=host_step)
+    req_e2e = int(sum_counters(np.array([d_e2e["n_requests"]], np.uint64))[0])
     h2d = Rp * wl.batch * 8
     d2h = Rp * wl.batch * 26 + 8 * len(STAT_NAMES)
 
@@ -273,7 +404,7 @@ def run_gpu(args):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms / K, "ms_per_step_repeat": ms_repeat / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u64 views, i64 ledgers, fp32 scores", "data": "synthetic",
             "config": {"workload": args.workload, "n_peers": st.n_peers, "n_replicas_per_gpu": Rp,
                        "requests_per_step_per_gpu": Rp * wl.batch, "batch_overridden": bool(args.batch), "flags": st.flags, "gossip_every": wl.gossip_every, "gossip_phase": "first timed step",
@@ -282,8 +413,9 @@ def run_gpu(args):
                               if 2 * 8 * st.n_peers ** 2 * Rp > 126e6 else
                               "inputs smaller than L2 and not flushed: this workload is a launch-latency case, not a bandwidth one")},
             "clocks": clocks,
-            "e2e": {"value": req_e2e / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / K, "entry": "wwws_step_host, pinned host buffers (mapped: the kernels read requests from and write results to them)"},
+            "sustained": sustained,
+            "e2e": {"value": req_e2e / (ms_e2e[0] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e[0] / K, "entry": "wwws_step_host, pinned host buffers"},
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_request_path": roof_req,
@@ -294,7 +426,13 @@ def run_gpu(args):
             "kernels": kernels,
             "step_mix": {k: delta[k] for k in ("n_requests", "n_delegated", "n_duel", "n_probes", "rounds")},
         }
-    net.close()
+    leg.close()
+    del io
+    # ---- the other large configurations, compactly (default run only) ---------------------------
+    if args.legs and args.workload == DEFAULT_WORKLOAD and not args.batch:
+        legs = [run_compact_leg(args, name, dev, world, rank, local) for name in EXTRA_LEGS]
+        if line is not None:
+            line["other_workloads"] = legs
     if world > 1:
         dist.destroy_process_group()
     return line
@@ -310,7 +448,7 @@ def oracle_run(workload, seed, steps, warmup, replicas=1, first_replica=0):
     o.bind_requests(wl.requests)
     s = 0
     for _ in range(warmup):
-        f, c, now, g = step_args(wl, s, warmup); o.run_step(f, c, now, g); s += 1
+        f, c, now, g = step_args(wl, s, warmup); o.run_step(f, c, now, g or s == 0); s += 1
     n0 = o.stats_dict()["n_requests"]
     t0 = time.perf_counter()
     for _ in range(steps):
@@ -318,15 +456,15 @@ def oracle_run(workload, seed, steps, warmup, replicas=1, first_replica=0):
     dt = time.perf_counter() - t0
     n = o.stats_dict()["n_requests"] - n0
     rounds = sum(1 for k in range(steps) if k % wl.gossip_every == 0)
-    desc = (f"{replicas} replica(s) of {workload}, {steps} steps of {wl.batch} requests with {rounds} gossip round(s), "
-            f"single thread")
+    desc = (f"{replicas} replica(s) of {workload}, {warmup} untimed step(s), then {steps} steps of {wl.batch} requests "
+            f"per replica with {rounds} gossip round(s), single thread")
     o.close()
     return n / dt, dt, desc
 
 
 def _oracle_worker(job):
     workload, seed, steps, replica = job
-    v, dt, _ = oracle_run(workload, seed, steps, 0, 1, replica)
+    v, dt, _ = oracle_run(workload, seed, steps, 1, 1, replica)
     return v * dt, dt
 
 
@@ -370,7 +508,15 @@ def run_reference(args):
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
 
-def main():
+def launcher_command(argv, n, port=None):
+    """The command that starts `n` ranks of this script on this node, one per GPU."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port or 29500 + os.getpid() % 2000), os.path.abspath(__file__)]
+    return cmd + list(argv)
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
@@ -381,12 +527,25 @@ def main():
     ap.add_argument("--push-pull", action="store_true", help="gossip as a full pairwise exchange (flag 8)")
     ap.add_argument("--greedy", action="store_true", help="greedy dispatch rule instead of the proportional draw (flag 4)")
     ap.add_argument("--batch", type=int, default=None, help="override requests per replica per step (saturation runs)")
+    ap.add_argument("--step-kernel", type=int, default=0, help="force the fused step's kernel (WWWS_OPT_STEP_KERNEL)")
+    ap.add_argument("--stream-run", type=int, default=0, help="requests per warp of the streaming kernel (WWWS_OPT_STREAM_RUN)")
+    ap.add_argument("--sustain-s", type=float, default=1.0, help="device seconds of the repeated timed region")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--no-legs", dest="legs", action="store_false", help="skip the compact legs on the other large workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing legs")
     ap.add_argument("--no-cpu-all-cores", action="store_true", help="skip the one-oracle-per-core timing leg")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be >= 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher yet: start one rank per GPU and let rank 0 print the line
+        if args.impl == "ours":
+            import torch
+            if torch.cuda.device_count() < args.gpus:
+                raise SystemExit(f"bench.py: --gpus {args.gpus} but {torch.cuda.device_count()} CUDA device(s) are visible")
+        raise SystemExit(subprocess.call(launcher_command(argv, args.gpus)))
     if args.impl == "reference":
         line = run_reference(args)
         if line:
@@ -396,14 +555,17 @@ def main():
     if line is not None:
         if args.gpus == 1 and not args.no_cpu_baseline:
             from paper_2603_20661_b200 import synth
-            ge = synth.make_workload(args.workload, n_replicas=1, n_requests=1000).gossip_every
-            v, dt, desc = oracle_run(args.workload, args.seed, ge, 0, 1)
+            wl = synth.make_workload(args.workload, n_requests=1000)
+            # the large networks are timed on two replicas (the cost is linear in replicas), the others on one
+            reps = 2 if wl.settings.n_replicas >= 2 and wl.settings.n_peers >= 2048 else 1
+            ge = wl.gossip_every
+            v, dt, desc = oracle_run(args.workload, args.seed, ge, 1, reps)
             if not args.no_cpu_all_cores:
                 try:
                     va, workers, wall = oracle_all_cores(args.workload, args.seed, ge)
                     line["cpu_baseline_all_cores"] = {
                         "value": va, "unit": UNIT, "cores": workers, "kind": "oracle", "wall_seconds": wall,
-                        "sample": f"{workers} independent oracle instances, one replica each, same steps"}
+                        "sample": f"{workers} independent oracle instances, one replica each, one untimed step, then the same steps"}
                 except Exception as e:          # a baseline leg must never cost the GPU result
                     line["cpu_baseline_all_cores"] = {"unavailable": repr(e)}
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,

@@ -129,16 +129,22 @@ __global__ void k_fold(Net n, int finalize_requested)
         if (db || finalize) refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], queued, credit_now);
     }
     if (finalize) {
+        // block sum of the committed credit, one atomic per block; the block that finishes a replica
+        // last commits it (no second launch): thread 0 makes its sum visible, then takes a ticket
+        __shared__ long long warp_sum[32];
         for (int o = 16; o; o >>= 1) csum += __shfl_down_sync(0xffffffffu, csum, o);
-        if ((threadIdx.x & 31) == 0 && csum) atomicAdd((unsigned long long*)&n.credit_check[r], (unsigned long long)csum);
-        // the block that finishes a replica last commits it (no second launch): every block makes
-        // its sums visible, then takes a ticket
-        __threadfence();
+        if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = csum;
         __syncthreads();
-        if (threadIdx.x == 0 && atomicAdd(&n.fold_ticket[r], 1u) == gridDim.x - 1) {
-            n.fold_ticket[r] = 0;
+        if (threadIdx.x == 0) {
+            long long bsum = 0;
+            for (uint32_t k = 0; k < (blockDim.x + 31) / 32; ++k) bsum += warp_sum[k];
+            if (bsum) atomicAdd((unsigned long long*)&n.credit_check[r], (unsigned long long)bsum);
             __threadfence();
-            finalize_replica(n, r);
+            if (atomicAdd(&n.fold_ticket[r], 1u) == gridDim.x - 1) {
+                n.fold_ticket[r] = 0;
+                __threadfence();
+                finalize_replica(n, r);
+            }
         }
     } else if (finalize_requested && blockIdx.x == 0 && threadIdx.x == 0) {
         n.stats[size_t(r) * sCount + sBlocksRejected] += 1;      // no majority: the block stays open

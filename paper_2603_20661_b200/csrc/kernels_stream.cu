@@ -49,9 +49,10 @@ struct alignas(16) WarpPool {
 
 struct Warp {                                  // warp-uniform scheduling state, in registers
     uint32_t sc_head, sc_n, dr_head, dr_n, vo_head, vo_n, fi_head, fi_n, n_free;
-    uint32_t next, end;                        // batch indices of the warp's requests not yet started
+    uint32_t chunk, n_chunks, stride, count;   // next 32-request chunk of the batch this warp starts; chunks go round the replica's warps
     uint32_t r, rg, lane, lt;                  // replica, global replica, lane, mask of the lower lanes
     uint64_t first;
+    size_t xbase, pbase;                       // replica's offset into the request arrays (+ first) and into the per-peer tables
 };
 
 // Counters of all the requests a thread finishes (a thread may finish hundreds).
@@ -81,19 +82,19 @@ __device__ __forceinline__ E4 ld_entries(const char* p)            // four view 
 template <bool SCORES>
 __device__ __forceinline__ void phase_origin(const Net& n, WarpPool& p, Warp& w)
 {
-    const uint32_t m = min(32u, w.end - w.next);
+    const uint32_t m = min(32u, w.count - 32u * w.chunk);
     const bool active = w.lane < m;
-    const uint32_t idx = w.next + w.lane;
+    const uint32_t idx = 32u * w.chunk + w.lane;
     bool offload = false;
     int code = -3;
     uint32_t where = 0;
     if (active) {
-        const size_t x = size_t(w.r) * n.Q + w.first + idx;
+        const size_t x = w.xbase + idx;
         const uint32_t o = n.origin[x];
         const Rnd4 rx = draw(n, uint32_t(w.first + idx), 0, w.rg, kOrigin);
         if (o >= n.N) set_error(n, eArg, o);
         else {
-            const uint32_t g = reinterpret_cast<const uint32_t*>(n.gate)[2 * (size_t(w.r) * n.N + o) + 1];
+            const uint32_t g = reinterpret_cast<const uint32_t*>(n.gate)[2 * (w.pbase + o) + 1];
             if (g & kGateOnline) {
                 code = (g & kGateNoCap) ? -4 : -1;
                 if (ppm(rx.w[0]) < (g & kGateFreq)) {
@@ -110,7 +111,7 @@ __device__ __forceinline__ void phase_origin(const Net& n, WarpPool& p, Warp& w)
     const uint32_t mo = __ballot_sync(kFull, offload), ml = __ballot_sync(kFull, active && !offload);
     if (offload) p.q_score[(w.sc_head + w.sc_n + __popc(mo & w.lt)) & (kQ - 1)] = make_uint2(idx, where);
     if (active && !offload) p.q_fin[(w.fi_head + w.fi_n + __popc(ml & w.lt)) & (kQ - 1)] = make_uint4(idx, uint32_t(code), 0xffffu, 0u);
-    w.sc_n += __popc(mo); w.fi_n += __popc(ml); w.next += m;
+    w.sc_n += __popc(mo); w.fi_n += __popc(ml); w.chunk += w.stride;
 }
 
 // ---- score: D4 ------------------------------------------------------------------------------------
@@ -130,20 +131,25 @@ __device__ __forceinline__ float candidate_score(const Net& n, bool not_self, ui
     return ok ? sc : 0.0f;
 }
 
+// The integer weight of a stored score: trunc(256 sc), at most 2^56 (the same value as weight_of()).
+__device__ __forceinline__ unsigned long long weight_q(float sc)
+{
+    return __float2ull_rz(fminf(__fmul_rn(sc, 256.0f), 72057594037927936.0f));
+}
+
 template <bool SCORES>
 __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, uint32_t m)
 {
     const bool active = w.lane < m;
-    uint32_t slot = 0;
     if (active) {
         const uint2 e = p.q_score[(w.sc_head + w.lane) & (kQ - 1)];
-        slot = p.free_slots[w.n_free - 1u - w.lane];
+        const uint32_t slot = p.free_slots[w.n_free - 1u - w.lane];
         const uint32_t o = e.y & 0xffffu, blk = (e.y >> 16) & 0x7ffu;
-        const char* row = reinterpret_cast<const char*>(n.view + (size_t(w.r) * n.N + o) * n.ld + kWin * blk);
+        const char* row = reinterpret_cast<const char*>(n.view + (w.pbase + o) * n.ld + kWin * blk);
         const float4* wl4 = reinterpret_cast<const float4*>(n.w_led + size_t(w.r) * n.ld + kWin * blk);
         const uint32_t self = (o >> 5) == blk ? (o & 31u) : 32u;
         float ssum = 0.0f;
-#pragma unroll
+#pragma unroll 1
         for (int h = 0; h < 2; ++h) {                                  // 16 candidates at a time: four 32-byte loads in flight
             E4 v[4];
             float4 f[4];
@@ -156,18 +162,19 @@ __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, 
                 unsigned long long gsum = 0;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const int k = 8 * g2 + j, c = 16 * h + k;
+                    const int k = 8 * g2 + j;
+                    const uint32_t c = 16u * h + k;
                     const float wl = (k & 3) == 0 ? f[k >> 2].x : (k & 3) == 1 ? f[k >> 2].y : (k & 3) == 2 ? f[k >> 2].z : f[k >> 2].w;
-                    const float sc = candidate_score(n, self != uint32_t(c), v[k >> 2].lo[k & 3], v[k >> 2].hi[k & 3], wl);
+                    const float sc = candidate_score(n, self != c, v[k >> 2].lo[k & 3], v[k >> 2].hi[k & 3], wl);
                     p.S[c][slot] = sc;
-                    gsum += weight_of(sc);
+                    gsum += weight_q(sc);
                     if (SCORES) ssum = __fadd_rn(ssum, sc);
                 }
                 p.G[2 * h + g2][slot] = gsum;
             }
         }
         p.ident[slot] = e.x; p.where[slot] = e.y; p.meta[slot] = 0u; p.picks[slot] = 0u;
-        if (SCORES && n.score_sum) n.score_sum[size_t(w.r) * n.Q + w.first + e.x] = ssum;
+        if (SCORES && n.score_sum) n.score_sum[w.xbase + e.x] = ssum;
         p.q_draw[(w.dr_head + w.dr_n + w.lane) & (kSlots - 1)] = uint8_t(slot);
     }
     w.sc_head += m; w.sc_n -= m; w.n_free -= m; w.dr_n += m;
@@ -190,25 +197,25 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
         uint32_t n_draws = meta & 0xffu, n_probes = (meta >> 8) & 0xffu, stage = (meta >> 16) & 3u, nj = (meta >> 18) & 7u;
         bool near = (meta >> 21) & 1u;
         const uint32_t blk = (where >> 16) & 0x7ffu, q = uint32_t(w.first + idx);
-        const size_t pbase = size_t(w.r) * n.N + kWin * blk;
+        const size_t cbase = w.pbase + kWin * blk;
         const unsigned long long G0 = p.G[0][slot], G1 = p.G[1][slot], G2 = p.G[2][slot], G3 = p.G[3][slot];
         const unsigned long long S = G0 + G1 + G2 + G3;
         int pick = -1;
         if (S != 0) {
             const uint32_t k = n_draws++;
-            int g;
+            uint32_t g;
             unsigned long long wp;
             if (GREEDY) {
                 // greedy rule: highest weight, lowest candidate on ties; flagged when the runner-up is within 1e-5
                 unsigned long long m1 = 0, m2 = 0;
-#pragma unroll 8
+#pragma unroll 4
                 for (int c = 0; c < int(kWin); ++c) {
-                    const unsigned long long x = weight_of(p.S[c][slot]);
+                    const unsigned long long x = weight_q(p.S[c][slot]);
                     if (x > m1) { m2 = m1; m1 = x; pick = c; }
                     else if (x > m2) m2 = x;
                 }
                 if (m2 != 0 && m1 - m2 <= m1 / 100000ull) near = true;
-                g = pick >> 3; wp = m1;
+                g = uint32_t(pick) >> 3; wp = m1;
             } else {
                 unsigned long long u;
                 if (k & 1u) u = p.ycache[slot];
@@ -218,24 +225,27 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
                     p.ycache[slot] = (unsigned long long)y.w[2] << 32 | y.w[3];
                 }
                 const unsigned long long r64 = __umul64hi(u, S);
-                unsigned long long lo = 0;
-                g = 0;
-                if (r64 >= G0) { lo = G0; g = 1;
-                    if (r64 >= lo + G1) { lo += G1; g = 2;
-                        if (r64 >= lo + G2) { lo += G2; g = 3; } } }
+                // the group whose interval holds r64, then the candidate inside it, without branches:
+                // the pick is the number of inclusive prefix sums that do not exceed r64
+                const unsigned long long c1 = G0 + G1, c2 = c1 + G2;
+                g = uint32_t(r64 >= G0) + uint32_t(r64 >= c1) + uint32_t(r64 >= c2);
+                unsigned long long lo = g == 0 ? 0ull : g == 1 ? G0 : g == 2 ? c1 : c2, acc = lo;
+                uint32_t cnt = 0;
                 wp = 0;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const unsigned long long x = weight_of(p.S[8 * g + j][slot]);
-                    if (pick < 0) {
-                        if (r64 < lo + x) { pick = 8 * g + j; wp = x; }
-                        else lo += x;
-                    }
+                    const unsigned long long x = weight_q(p.S[8 * g + j][slot]);
+                    const bool below = acc + x <= r64;                   // candidate j ends at or before r64
+                    if (!below && cnt == uint32_t(j)) wp = x;            // the first one that does not is the pick
+                    acc += x;
+                    if (below) { lo = acc; ++cnt; }
                 }
+                pick = int(8u * g + cnt);
                 const unsigned long long d1 = r64 - lo, d2 = lo + wp - 1 - r64;
                 if ((d1 < d2 ? d1 : d2) <= S / 100000ull) near = true;
+                if (cnt >= 8u) pick = -1;                                // cannot happen: the group sums are the sums of the weights in play
             }
-            if (pick >= 0) {                                            // always: the group sums are the sums of the weights in play
+            if (pick >= 0) {
                 if (SCORES && stage == 0 && n.score_a) fin.x = __float_as_uint(p.S[pick][slot]);     // the executor's score, if this pick accepts
                 p.S[pick][slot] = 0.0f;
                 p.G[g][slot] = (g == 0 ? G0 : g == 1 ? G1 : g == 2 ? G2 : G3) - wp;
@@ -246,20 +256,20 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
         else if (stage < 2) {
             ++n_probes;
             // D6: the drawn candidate answers by its true state and its own accept policy (its gate)
-            const uint32_t thr = reinterpret_cast<const uint32_t*>(n.gate)[2 * (pbase + pick)];
+            const uint32_t thr = reinterpret_cast<const uint32_t*>(n.gate)[2 * (cbase + pick)];
             const Rnd4 y = draw(n, q, uint32_t(pick) >> 2, w.rg, kProbe);
             const uint32_t sel = uint32_t(pick) & 3u;
             const bool accepted = ppm(sel == 0 ? y.w[0] : sel == 1 ? y.w[1] : sel == 2 ? y.w[2] : y.w[3]) < thr;
             if (accepted) {
                 if (stage == 0) {
                     picks = uint32_t(pick);
-                    if (SCORES && n.score_a) n.score_a[size_t(w.r) * n.Q + w.first + idx] = __uint_as_float(fin.x);
+                    if (SCORES && n.score_a) n.score_a[w.xbase + idx] = __uint_as_float(fin.x);
                     if (where & kWhereDuel) { stage = 1; if (n_probes >= n.max_probes) kind = kFinCancel; }
                     else kind = kFinPlain;
                 } else { picks |= uint32_t(pick) << 5; stage = 2; }
             } else if (n_probes >= n.max_probes) kind = stage == 0 ? kFinNone : kFinCancel;
         } else {
-            if (n.online[pbase + pick]) { picks |= uint32_t(pick) << (10u + 5u * nj); ++nj; }
+            if (n.online[cbase + pick]) { picks |= uint32_t(pick) << (10u + 5u * nj); ++nj; }
             if (nj >= n.n_judges) kind = kVote;
         }
         if (kind == kCont || kind == kVote) {
@@ -293,13 +303,13 @@ __device__ __forceinline__ void phase_vote(const Net& n, WarpPool& p, Warp& w, u
         const uint32_t meta = p.meta[slot], where = p.where[slot], idx = p.ident[slot], picks = p.picks[slot];
         const uint32_t blk = (where >> 16) & 0x7ffu, o = where & 0xffffu, q = uint32_t(w.first + idx);
         const uint32_t nj = (meta >> 18) & 7u;
-        const size_t pbase = size_t(w.r) * n.N;
         const int a = int(kWin * blk + (picks & 31u)), b = int(kWin * blk + ((picks >> 5) & 31u));
         int jd[4];
 #pragma unroll
         for (int l = 0; l < 4; ++l) jd[l] = uint32_t(l) < nj ? int(kWin * blk + ((picks >> (10 + 5 * l)) & 31u)) : -1;
-        const unsigned long long thr = ((1ull << 32) + n.quality[pbase + a] - n.quality[pbase + b]) >> 1;
+        const unsigned long long thr = ((1ull << 32) + n.quality[w.pbase + a] - n.quality[w.pbase + b]) >> 1;
         uint32_t votes_a = 0;
+#pragma unroll 1
         for (uint32_t l = 0; l < nj; ++l) {
             const Rnd4 y = draw(n, q, l, w.rg, kJudge);
             bool va = (unsigned long long)y.w[0] < thr;
@@ -307,9 +317,9 @@ __device__ __forceinline__ void phase_vote(const Net& n, WarpPool& p, Warp& w, u
             votes_a += va;
         }
         const uint32_t oc = 2u * votes_a > nj ? 1u : (2u * votes_a < nj ? 2u : 3u);
-        const size_t x = size_t(w.r) * n.Q + w.first + idx;
+        const size_t x = w.xbase + idx;
         const long long extra = settle_duel(n, w.r, q, o, n.len_in[x], n.len_out[x], a, b, jd, oc, acc);
-        add64(&n.d_credit[pbase + o], -extra);
+        add64(&n.d_credit[w.pbase + o], -extra);
         p.q_fin[(w.fi_head + w.fi_n + w.lane) & (kQ - 1)] =
             make_uint4(idx, uint32_t(a), uint32_t(b) | blk << 16,
                        ((picks >> 10) & 0xfffffu) | nj << 20 | oc << 23 | ((meta >> 21) & 1u) << 26 | ((meta >> 8) & 15u) << 27);
@@ -329,7 +339,7 @@ __device__ __forceinline__ void phase_finish(const Net& n, WarpPool& p, Warp& w,
         int jd[4];
 #pragma unroll
         for (int l = 0; l < 4; ++l) jd[l] = uint32_t(l) < nj ? int(kWin * blk + ((e.w >> (5 * l)) & 31u)) : -1;
-        const size_t x = size_t(w.r) * n.Q + w.first + idx;
+        const size_t x = w.xbase + idx;
         n.exec_a[x] = a; n.exec_b[x] = b; n.outcome[x] = uint8_t(oc); n.rflags[x] = near ? 1 : 0;
         *reinterpret_cast<int4*>(n.judges + 4 * x) = make_int4(jd[0], jd[1], jd[2], jd[3]);
         acc.probes += e.w >> 27;
@@ -339,15 +349,18 @@ __device__ __forceinline__ void phase_finish(const Net& n, WarpPool& p, Warp& w,
     w.fi_head += m; w.fi_n -= m;
 }
 
+enum : int { phOrigin, phScore, phDraw, phVote, phFinish, phDone };
+
 template <bool GREEDY, bool SCORES>
-__global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, uint32_t count, uint32_t per_warp)
+__global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, uint32_t count)
 {
     __shared__ WarpPool p;
     Warp w;
     w.lane = threadIdx.x; w.lt = (1u << w.lane) - 1u;
     w.r = blockIdx.y; w.rg = w.r + n.replica_offset; w.first = first;
-    w.next = blockIdx.x * per_warp;
-    w.end = min(count, w.next + per_warp);
+    w.xbase = size_t(w.r) * n.Q + first; w.pbase = size_t(w.r) * n.N;
+    w.count = count; w.n_chunks = (count + 31u) / 32u;
+    w.chunk = blockIdx.x; w.stride = gridDim.x;
     w.sc_head = w.sc_n = w.dr_head = w.dr_n = w.vo_head = w.vo_n = w.fi_head = w.fi_n = 0;
     w.n_free = kSlots;
     p.free_slots[w.lane] = uint8_t(w.lane); p.free_slots[w.lane + 32] = uint8_t(w.lane + 32);
@@ -358,25 +371,35 @@ __global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, u
 
     // A phase runs when 32 requests wait for it, later phases first (queues stay short and never
     // overflow: whatever feeds the finish queue runs only while it holds fewer than 32 entries,
-    // and the score queue is fed only while it holds fewer than 32).
+    // and the score queue is fed only while it holds fewer than 32).  Each phase's code exists once.
+#pragma unroll 1
     for (;;) {
-        __syncwarp();
-        if (w.fi_n >= 32u) { phase_finish(n, p, w, 32u, acc); continue; }
-        if (w.vo_n >= 32u) { phase_vote(n, p, w, 32u, acc); continue; }
-        if (w.dr_n >= 32u) { phase_draw<GREEDY, SCORES>(n, p, w, 32u); continue; }
-        if (w.sc_n >= 32u) {
-            if (w.n_free >= 32u) { phase_score<SCORES>(n, p, w, 32u); continue; }
+        int ph = phDone;
+        uint32_t m = 32u;
+        if (w.fi_n >= 32u) ph = phFinish;
+        else if (w.vo_n >= 32u) ph = phVote;
+        else if (w.dr_n >= 32u) ph = phDraw;
+        else if (w.sc_n >= 32u) {
+            if (w.n_free >= 32u) ph = phScore;
             // all windows taken: the draw and vote queues hold more than 32 between them, so the longer is at least half a warp
-            if (w.dr_n >= w.vo_n) phase_draw<GREEDY, SCORES>(n, p, w, w.dr_n); else phase_vote(n, p, w, w.vo_n, acc);
-            continue;
+            else if (w.dr_n >= w.vo_n) { ph = phDraw; m = w.dr_n; }
+            else { ph = phVote; m = w.vo_n; }
         }
-        if (w.next < w.end) { phase_origin<SCORES>(n, p, w); continue; }
+        else if (w.chunk < w.n_chunks) ph = phOrigin;
         // input exhausted: what is left runs in partial batches, earlier phases first so that the later ones fill up
-        if (w.sc_n && w.n_free) { phase_score<SCORES>(n, p, w, min(w.sc_n, w.n_free)); continue; }
-        if (w.dr_n) { phase_draw<GREEDY, SCORES>(n, p, w, w.dr_n); continue; }
-        if (w.vo_n) { phase_vote(n, p, w, w.vo_n, acc); continue; }
-        if (w.fi_n) { phase_finish(n, p, w, w.fi_n, acc); continue; }
-        break;
+        else if (w.sc_n && w.n_free) { ph = phScore; m = min(w.sc_n, w.n_free); }
+        else if (w.dr_n) { ph = phDraw; m = w.dr_n; }
+        else if (w.vo_n) { ph = phVote; m = w.vo_n; }
+        else if (w.fi_n) { ph = phFinish; m = w.fi_n; }
+        if (ph == phDone) break;
+        __syncwarp();
+        switch (ph) {
+        case phOrigin: phase_origin<SCORES>(n, p, w); break;
+        case phScore: phase_score<SCORES>(n, p, w, m); break;
+        case phDraw: phase_draw<GREEDY, SCORES>(n, p, w, m); break;
+        case phVote: phase_vote(n, p, w, m, acc); break;
+        default: phase_finish(n, p, w, m, acc); break;
+        }
     }
 
     // counters: one warp reduction and one atomic per counter
@@ -395,30 +418,42 @@ __global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, u
     }
 }
 
-// Requests per warp: enough warps to fill the GPU (about 12 per SM) first, then longer runs per
-// warp, which is what lets the phases run full; WWWS_OPT_STREAM_RUN overrides it.
-uint32_t stream_requests_per_warp(uint64_t total)
+// Warps per replica: all warps of the launch are resident at once (one wave: no tail), and a
+// replica's 32-request chunks go round its warps, so every warp gets the same number of them
+// (give or take one).  More chunks per warp is what lets the phases run full.
+// `run` (WWWS_OPT_STREAM_RUN) instead fixes the requests per warp.
+static uint32_t stream_warps_per_replica(const Net& n, uint32_t count, uint32_t run, int resident_warps)
 {
-    const uint64_t warps = 148ull * 12;
-    uint64_t per = (total + warps - 1) / warps;
-    per = (per + 31) / 32 * 32;
-    if (per < 64) per = 64;
-    if (per > 512) per = 512;
-    return uint32_t(per);
+    const uint32_t chunks = (count + 31u) / 32u;
+    uint32_t g = run ? (count + run - 1u) / run : uint32_t(resident_warps) / n.Rp;
+    if (g < 1u) g = 1u;
+    return g > chunks ? chunks : g;
 }
 
-void launch_step_stream(const Net& n, uint64_t first, uint32_t count, uint32_t per_warp, const LaunchCtx& c)
+template <bool GREEDY, bool SCORES>
+static void launch_stream_variant(const Net& n, uint64_t first, uint32_t count, uint32_t run, const LaunchCtx& c)
+{
+    static const int resident = [] {
+        int dev = 0, sms = 0, per_sm = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_step_stream<GREEDY, SCORES>, 32, 0);
+        return sms * per_sm > 0 ? sms * per_sm : 148 * 15;
+    }();
+    const dim3 grid(stream_warps_per_replica(n, count, run, resident), n.Rp);
+    k_step_stream<GREEDY, SCORES><<<grid, 32, 0, c.stream>>>(n, first, count);
+}
+
+void launch_step_stream(const Net& n, uint64_t first, uint32_t count, uint32_t run, const LaunchCtx& c)
 {
     Timed t(c, kStepFused);
-    if (per_warp == 0) per_warp = stream_requests_per_warp(uint64_t(count) * n.Rp);
-    const dim3 grid((count + per_warp - 1) / per_warp, n.Rp);
     const bool scores = n.score_a || n.score_sum;
     if (n.flags & 4u) {
-        if (scores) k_step_stream<true, true><<<grid, 32, 0, c.stream>>>(n, first, count, per_warp);
-        else k_step_stream<true, false><<<grid, 32, 0, c.stream>>>(n, first, count, per_warp);
+        if (scores) launch_stream_variant<true, true>(n, first, count, run, c);
+        else launch_stream_variant<true, false>(n, first, count, run, c);
     } else {
-        if (scores) k_step_stream<false, true><<<grid, 32, 0, c.stream>>>(n, first, count, per_warp);
-        else k_step_stream<false, false><<<grid, 32, 0, c.stream>>>(n, first, count, per_warp);
+        if (scores) launch_stream_variant<false, true>(n, first, count, run, c);
+        else launch_stream_variant<false, false>(n, first, count, run, c);
     }
 }
 

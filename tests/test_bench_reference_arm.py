@@ -41,3 +41,32 @@ def test_step_schedule_and_byte_model():
     assert (f2, c2) == (0, wl.batch) and now2 > bench.step_args(wl, n - 1)[2]
     g, r = bench.algorithmic_bytes(wl, {"n_requests": 10, "n_delegated": 4, "n_fallback_local": 1, "n_failed": 0})
     assert g == 2 * 8 * 8 * 8 and r == 10 * 34 + 5 * 256
+
+
+def test_gpus_2_starts_two_ranks_and_rank_0_prints_the_line():
+    """`--gpus 2` outside a launcher starts two processes itself (one per GPU for the GPU arm); with
+    the reference arm only rank 0 works and prints."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload", "tiny",
+                          "--steps", "4", "--warmup", "3"], capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip().startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
+
+
+def test_launcher_command_and_missing_devices():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launcher_command(["--gpus", "4", "--steps", "2"], 4, port=29555)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29555"
+    assert cmd[-5] == os.path.join(ROOT, "bench.py") and cmd[-4:] == ["--gpus", "4", "--steps", "2"]
+    import torch
+    if torch.cuda.device_count() < 2:
+        # fewer devices than ranks: a clear refusal, not a silent single-GPU timing
+        env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+        out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--workload", "tiny"],
+                             capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
+        assert out.returncode != 0 and "--gpus 2" in out.stderr and out.stdout.strip() == ""
