@@ -46,7 +46,10 @@ typedef enum {
     WWWS_ERR_RANGE = 4,     /* a peer's version counter reached 2^24 */
     WWWS_ERR_CUDA = 5,      /* a CUDA runtime call failed */
     WWWS_ERR_INVARIANT = 6, /* total credit changed across a settlement */
-    WWWS_ERR_TIMEOUT = 7    /* reserved */
+    WWWS_ERR_TIMEOUT = 7,   /* reserved */
+    WWWS_ERR_INDEX = 8      /* only from a library built with -DWWWS_CHECK_INDICES: an index that a kernel took from
+                               device data (a partner id, a list offset, a candidate or executor id) was out of
+                               range; the access was skipped and the results of that call are not to be trusted */
 } wwws_status;
 
 #define WWWS_WINDOW 32u      /* candidate-window width: peers per block of the id ring */
@@ -227,11 +230,13 @@ typedef struct {
 } wwws_host_io;
 
 /* wwws_step with HOST buffers; synchronises before it returns.  totals_out (HOST, one record) may be NULL.
- * If all eight buffers are page-locked and mapped into the device's address space (cudaHostAlloc,
- * cudaHostRegister) and exact queueing (WWWS_FLAG_FIFO) is off, the kernels read the batch's requests
- * from, and write its results to, the host buffers directly; the bound device arrays are not touched.
- * Otherwise the batch's request slices are copied to the bound device arrays, the step runs on
- * those, and the batch's results are copied back.  Either way the total counters come back in totals_out. */
+ * Two ways, with identical results.  Direct: if all eight buffers are page-locked and mapped into the device's
+ * address space (cudaHostAlloc, cudaHostRegister), exact queueing (WWWS_FLAG_FIFO) is off and the batch is small
+ * (n_replicas * count <= 16384, or WWWS_OPT_HOST_IO = 1), the kernels read the batch's requests from, and write
+ * its results to, the host buffers themselves; the bound device arrays are not touched.  Staged: the batch's
+ * request slices are copied to the bound device arrays on a second stream (created at the first such call)
+ * while time advance and gossip run, the step runs on the device arrays, and the batch's results are copied
+ * back on that stream while the block is folded.  Either way the total counters come back in totals_out. */
 wwws_status wwws_step_host(wwws_network* net, const wwws_host_io* io, uint64_t first, uint64_t count,
                            uint32_t now_ms, int do_gossip, int finalize, wwws_stats_t* totals_out);
 
@@ -271,8 +276,16 @@ typedef enum {
                                    1 eight lanes per request, 2 four lanes per request, 3 one thread per request,
                                    4 streaming phases (a warp takes a run of requests through origin / score /
                                    draw / vote / finish with full warps) */
-    WWWS_OPT_STREAM_RUN = 2     /* requests per warp of the streaming kernel: 0 chosen by launch size (default),
+    WWWS_OPT_STREAM_RUN = 2,    /* requests per warp of the streaming kernel: 0 chosen by launch size (default),
                                    else a multiple of 32 */
+    WWWS_OPT_HOST_IO = 4,       /* wwws_step_host: 0 (default) chosen by batch size, 1 kernels read and write mapped host
+                                   buffers directly where possible, 2 always staged copies */
+    WWWS_OPT_LAUNCH_OVERLAP = 3 /* mask of the kernels that are launched so that their grid may be scheduled while the
+                                   previous grid of the stream finishes (programmatic dependent launch; every kernel
+                                   waits for its predecessor's completion before it touches memory): bit 0 time
+                                   advance and the rest, bit 1 gossip, bit 2 request kernels, bit 3 fold.  Default: 15
+                                   for networks of up to 32,768 peer-replicas (their steps are chains of launch
+                                   latencies), 0 for larger ones */
 } wwws_option;
 wwws_status wwws_set_option(wwws_network* net, wwws_option option, int64_t value);
 

@@ -14,10 +14,10 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SO = os.path.join(_HERE, "libwwws.so")
+_SO = os.environ.get("WWWS_LIBRARY") or os.path.join(_HERE, "libwwws.so")     # e.g. the index-checked build
 
 STATUS = {0: "OK", 1: "ERR_ARG", 2: "ERR_ALLOC", 3: "ERR_STATE", 4: "ERR_RANGE", 5: "ERR_CUDA", 6: "ERR_INVARIANT",
-          7: "ERR_TIMEOUT"}
+          7: "ERR_TIMEOUT", 8: "ERR_INDEX"}
 STAT_NAMES = ("n_requests", "n_local", "n_fallback_local", "n_dropped", "n_failed", "n_delegated", "n_duel",
               "n_duel_cancelled", "n_draw", "n_judge_evals", "n_probes", "n_near_boundary", "slo_met",
               "sum_latency_ms", "n_offline_marks", "rounds", "blocks", "credit_total", "chain_head", "pending_digest", "n_uncovered", "blocks_rejected")

@@ -29,7 +29,15 @@ struct wwws_network {
     uint64_t launches;
     Profiler prof;
     std::string err;
-    LaunchCtx ctx() { return LaunchCtx{ stream, &launches, &prof }; }
+    int host_io = 0;             // wwws_step_host: 0 by batch size, 1 kernels use mapped host buffers, 2 staged copies
+    cudaStream_t copy_stream = nullptr;          // staged host path: copies run beside the kernels
+    cudaEvent_t ev_fork = nullptr, ev_in = nullptr, ev_step = nullptr;
+    int overlap = 0;             // which launches may overlap their predecessor's tail (WWWS_OPT_LAUNCH_OVERLAP):
+                                 // bit 0 time advance, 1 gossip, 2 request kernels, 3 fold; other kernels follow bit 0.
+                                 // Set at creation: all for small networks, whose steps are a chain of launch latencies;
+                                 // none for large ones, where a chain of early-resident waiting grids slowed the step down
+                                 // (1,024 peers x 256 replicas: 0.47 ms per step plain, 0.61 ms with every launch overlapped)
+    LaunchCtx ctx(int kind = 1) { return LaunchCtx{ stream, &launches, &prof, (overlap & kind) != 0 && !prof.enabled }; }
     struct TableInfo { void* ptr; uint32_t elem; } tables[WWWS_T_COUNT];
 };
 
@@ -156,6 +164,7 @@ wwws_status check_device_error(wwws_network* n)
     case eRange: snprintf(buf, sizeof buf, "version counter of peer %u reached 2^24", e[1]); return fail(n, WWWS_ERR_RANGE, buf);
     case eInvariant: snprintf(buf, sizeof buf, "total credit of replica %u changed across finalization", e[1]); return fail(n, WWWS_ERR_INVARIANT, buf);
     case eArg: snprintf(buf, sizeof buf, "request with origin index %u >= n_peers (dropped)", e[1]); return fail(n, WWWS_ERR_ARG, buf);
+    case eIndex: snprintf(buf, sizeof buf, "checked build: an index taken from device data was out of range at site %u (access skipped)", e[1]); return fail(n, WWWS_ERR_INDEX, buf);
     default: snprintf(buf, sizeof buf, "device error word %u/%u", e[0], e[1]); return fail(n, WWWS_ERR_CUDA, buf);
     }
 }
@@ -221,6 +230,7 @@ wwws_status wwws_create_network(const wwws_config* cfg, const wwws_peer_init* in
     if (cv.off > workspace_bytes) return fail(nullptr, WWWS_ERR_ALLOC, "workspace too small");
     n->cfg = *cfg; n->cfg.rank_cdf = nullptr;
     n->stream = static_cast<cudaStream_t>(cuda_stream);
+    n->overlap = uint64_t(cfg->n_peers) * cfg->n_replicas <= 32768 ? 15 : 0;
     n->ws = static_cast<uint8_t*>(workspace); n->ws_bytes = workspace_bytes;
     Net& d = n->d;
     d.N = cfg->n_peers; d.Rp = cfg->n_replicas; d.ld = (d.N + kWin - 1) / kWin * kWin; d.n_blk = d.ld / kWin;
@@ -285,6 +295,11 @@ wwws_status wwws_destroy_network(wwws_network* n)
     {
         DeviceScope scope(n->device);
         cudaStreamSynchronize(n->stream);
+        if (n->copy_stream) {
+            cudaStreamSynchronize(n->copy_stream);
+            cudaEventDestroy(n->ev_fork); cudaEventDestroy(n->ev_in); cudaEventDestroy(n->ev_step);
+            cudaStreamDestroy(n->copy_stream);
+        }
     }
     delete n;
     return WWWS_OK;
@@ -382,22 +397,32 @@ wwws_status wwws_settle_credits(wwws_network* n, int finalize)
     return launch_status(n, "settle_credits");
 }
 
+// One step; `inputs_ready` (may be null) is waited for before the request kernel, `results_ready`
+// (may be null) is recorded right after it: the staged host path copies beside the other kernels.
+static wwws_status step_impl(wwws_network* n, uint64_t first, uint64_t count, uint32_t now_ms, int do_gossip, int finalize,
+                             cudaEvent_t inputs_ready, cudaEvent_t results_ready)
+{
+    launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx(1));
+    n->t_last_ms = now_ms;
+    if (do_gossip) {
+        launch_gossip(n->d, n->round, n->ctx(2));
+        std::swap(n->d.view, n->d.view_new);
+        n->round += 1;
+    }
+    if (inputs_ready) CUDA_TRY(n, cudaStreamWaitEvent(n->stream, inputs_ready, 0));
+    launch_step_fused(n->d, first, uint32_t(count), n->ctx(4), n->step_kernel, n->stream_run);
+    if (results_ready) CUDA_TRY(n, cudaEventRecord(results_ready, n->stream));
+    if (n->d.flags & 16u) launch_fifo(n->d, first, uint32_t(count), n->ctx(4));
+    launch_fold(n->d, finalize != 0, n->ctx(8));
+    return launch_status(n, "step");
+}
+
 wwws_status wwws_step(wwws_network* n, uint64_t first, uint64_t count, uint32_t now_ms, int do_gossip, int finalize)
 {
     if (wwws_status st = check_batch(n, first, count)) return st;
     if (now_ms < n->t_last_ms) return fail(n, WWWS_ERR_ARG, "time must not go back");
     ON_DEVICE(n);
-    launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx());
-    n->t_last_ms = now_ms;
-    if (do_gossip) {
-        launch_gossip(n->d, n->round, n->ctx());
-        std::swap(n->d.view, n->d.view_new);
-        n->round += 1;
-    }
-    launch_step_fused(n->d, first, uint32_t(count), n->ctx(), n->step_kernel, n->stream_run);
-    if (n->d.flags & 16u) launch_fifo(n->d, first, uint32_t(count), n->ctx());
-    launch_fold(n->d, finalize != 0, n->ctx());
-    return launch_status(n, "step");
+    return step_impl(n, first, count, now_ms, do_gossip, finalize, nullptr, nullptr);
 }
 
 wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t first, uint64_t count, uint32_t now_ms,
@@ -407,7 +432,12 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
     if (!io || !io->origin || !io->len_in || !io->len_out || !io->exec_a || !io->exec_b || !io->judges || !io->outcome || !io->flags)
         return fail(n, WWWS_ERR_ARG, "a host buffer is NULL");
     ON_DEVICE(n);
-    if (!(n->d.flags & 16u)) {
+    if (now_ms < n->t_last_ms) return fail(n, WWWS_ERR_ARG, "time must not go back");
+    // Large batches go through staged copies even when the buffers are mapped: result records written
+    // across the bus request by request, in the order the kernel finishes them, cost more than three
+    // strided copies that run beside the kernels.
+    const bool want_direct = n->host_io == 1 || (n->host_io == 0 && count * n->d.Rp <= 16384);
+    if (!(n->d.flags & 16u) && want_direct) {
         // Page-locked, mapped host buffers are read and written by the kernels themselves: no copies,
         // and the result stores travel while the step runs.  (With exact queueing the results are
         // read again by later kernels, which is better done from device memory.)
@@ -428,7 +458,7 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
             d.exec_a = static_cast<int32_t*>(dev[3]); d.exec_b = static_cast<int32_t*>(dev[4]); d.judges = static_cast<int32_t*>(dev[5]);
             d.outcome = static_cast<uint8_t*>(dev[6]); d.rflags = static_cast<uint8_t*>(dev[7]);
             d.score_a = nullptr; d.score_sum = nullptr;
-            const wwws_status st = wwws_step(n, first, count, now_ms, do_gossip, finalize);
+            const wwws_status st = step_impl(n, first, count, now_ms, do_gossip, finalize, nullptr, nullptr);
             d.origin = saved.origin; d.len_in = saved.len_in; d.len_out = saved.len_out;
             d.exec_a = saved.exec_a; d.exec_b = saved.exec_b; d.judges = saved.judges; d.outcome = saved.outcome; d.rflags = saved.rflags;
             d.score_a = saved.score_a; d.score_sum = saved.score_sum;
@@ -442,28 +472,42 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
             return check_device_error(n);
         }
     }
+    // Staged path: the batch's request slices go to the bound device arrays on a second stream while
+    // time advance and gossip run; the request kernel waits for them; the results travel back on the
+    // second stream while the block is folded and the counters are read.
+    if (!n->copy_stream) {
+        CUDA_TRY(n, cudaStreamCreateWithFlags(&n->copy_stream, cudaStreamNonBlocking));
+        CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_fork, cudaEventDisableTiming));
+        CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_in, cudaEventDisableTiming));
+        CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_step, cudaEventDisableTiming));
+    }
     const Net& d = n->d;
-    cudaStream_t s = n->stream;
+    cudaStream_t cs = n->copy_stream;
     const size_t Q = d.Q, Rp = d.Rp, c = count;
     // the batch is one strided slice per array: Rp rows of `count` elements, pitch n_requests
-#define COPY2D(dst, src, T, W, kind) CUDA_TRY(n, cudaMemcpy2DAsync((void*)((dst) + first * (W)), Q * sizeof(T) * (W), (src) + first * (W), Q * sizeof(T) * (W), c * sizeof(T) * (W), Rp, kind, s))
+#define COPY2D(dst, src, T, W, kind) CUDA_TRY(n, cudaMemcpy2DAsync((void*)((dst) + first * (W)), Q * sizeof(T) * (W), (src) + first * (W), Q * sizeof(T) * (W), c * sizeof(T) * (W), Rp, kind, cs))
+    CUDA_TRY(n, cudaEventRecord(n->ev_fork, n->stream));               // whatever still reads the device arrays comes first
+    CUDA_TRY(n, cudaStreamWaitEvent(cs, n->ev_fork, 0));
     COPY2D(d.origin, io->origin, uint32_t, 1, cudaMemcpyHostToDevice);
     COPY2D(d.len_in, io->len_in, uint16_t, 1, cudaMemcpyHostToDevice);
     COPY2D(d.len_out, io->len_out, uint16_t, 1, cudaMemcpyHostToDevice);
-    if (wwws_status st = wwws_step(n, first, count, now_ms, do_gossip, finalize)) return st;
+    CUDA_TRY(n, cudaEventRecord(n->ev_in, cs));
+    if (wwws_status st = step_impl(n, first, count, now_ms, do_gossip, finalize, n->ev_in, n->ev_step)) { cudaStreamSynchronize(cs); return st; }
+    CUDA_TRY(n, cudaStreamWaitEvent(cs, n->ev_step, 0));
     COPY2D(io->exec_a, d.exec_a, int32_t, 1, cudaMemcpyDeviceToHost);
     COPY2D(io->exec_b, d.exec_b, int32_t, 1, cudaMemcpyDeviceToHost);
     COPY2D(io->judges, d.judges, int32_t, 4, cudaMemcpyDeviceToHost);
     COPY2D(io->outcome, d.outcome, uint8_t, 1, cudaMemcpyDeviceToHost);
     COPY2D(io->flags, d.rflags, uint8_t, 1, cudaMemcpyDeviceToHost);
 #undef COPY2D
+    wwws_status st = WWWS_OK;
     if (totals_out) {
         std::vector<wwws_stats_t> all(Rp + 1);
-        if (wwws_status st = wwws_stats(n, all.data())) return st;
-        *totals_out = all[Rp];
-        return WWWS_OK;
-    }
-    return check_device_error(n);
+        st = wwws_stats(n, all.data());
+        if (!st) *totals_out = all[Rp];
+    } else st = check_device_error(n);
+    CUDA_TRY(n, cudaStreamSynchronize(cs));
+    return st;
 }
 
 wwws_status wwws_stats(wwws_network* n, wwws_stats_t* host_out)
@@ -574,6 +618,14 @@ wwws_status wwws_set_option(wwws_network* n, wwws_option option, int64_t value)
     case WWWS_OPT_STEP_KERNEL:
         if (value < 0 || value > 4) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_STEP_KERNEL takes 0 (by size), 1 (8 lanes), 2 (4 lanes), 3 (thread) or 4 (streaming)");
         n->step_kernel = int(value);
+        return WWWS_OK;
+    case WWWS_OPT_HOST_IO:
+        if (value < 0 || value > 2) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_HOST_IO takes 0 (by batch size), 1 (mapped buffers) or 2 (staged copies)");
+        n->host_io = int(value);
+        return WWWS_OK;
+    case WWWS_OPT_LAUNCH_OVERLAP:
+        if (value < 0 || value > 15) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_LAUNCH_OVERLAP takes a mask 0..15");
+        n->overlap = int(value);
         return WWWS_OK;
     case WWWS_OPT_STREAM_RUN:
         if (value < 0 || value > 65536 || value % 32) return fail(n, WWWS_ERR_ARG, "WWWS_OPT_STREAM_RUN takes 0 (by size) or a multiple of 32 up to 65536");

@@ -9,6 +9,7 @@ namespace wwws {
 // G0 churn, G1 new version of the own entry, partner choice of G2 (reads the old view only).
 __global__ void k_gossip_peer(Net n, uint32_t round)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n.N) return;
     const uint32_t rg = r + n.replica_offset;
@@ -36,7 +37,7 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
                 const uint32_t p = below(g.w[s], n.N);
                 if (p == i) continue;
                 const uint64_t e = row[p];
-                if (e != 0 && !(e & kOffBit)) { part[s] = int32_t(p); open &= ~(1u << s); }
+                if (e != 0 && !(e & kOffBit) && index_ok(n, p, n.N, 101)) { part[s] = int32_t(p); open &= ~(1u << s); }
             }
         }
     }
@@ -50,15 +51,16 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
 // p >= 0 = answered, -2 - p = chosen but dead, -1 = no partner in that slot.
 __global__ void k_gossip_resolve(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n.N) return;
     const size_t x = size_t(r) * n.N + i;
     int4 p4 = *reinterpret_cast<const int4*>(n.partner + x * 4);
     const uint8_t* on = n.online + size_t(r) * n.N;
-    if (p4.x >= 0 && !on[p4.x]) p4.x = -2 - p4.x;
-    if (p4.y >= 0 && !on[p4.y]) p4.y = -2 - p4.y;
-    if (p4.z >= 0 && !on[p4.z]) p4.z = -2 - p4.z;
-    if (p4.w >= 0 && !on[p4.w]) p4.w = -2 - p4.w;
+    if (p4.x >= 0) { if (!index_ok(n, p4.x, n.N, 102)) p4.x = -1; else if (!on[p4.x]) p4.x = -2 - p4.x; }
+    if (p4.y >= 0) { if (!index_ok(n, p4.y, n.N, 102)) p4.y = -1; else if (!on[p4.y]) p4.y = -2 - p4.y; }
+    if (p4.z >= 0) { if (!index_ok(n, p4.z, n.N, 102)) p4.z = -1; else if (!on[p4.z]) p4.z = -2 - p4.z; }
+    if (p4.w >= 0) { if (!index_ok(n, p4.w, n.N, 102)) p4.w = -1; else if (!on[p4.w]) p4.w = -2 - p4.w; }
     *reinterpret_cast<int4*>(n.partner + x * 4) = p4;
 }
 
@@ -107,6 +109,7 @@ template <bool PUSH>
 __global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Net n, uint32_t panel_cols, uint32_t chunk_shift,
                                                                      uint32_t n_panels, uint32_t groups_per_panel)
 {
+    grid_dependency_enter();
     const uint32_t b = blockIdx.x;
     const uint32_t per_replica = n_panels * groups_per_panel;
     const uint32_t r = b / per_replica;
@@ -132,7 +135,13 @@ __global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Ne
     for (int it = 0; it < kMergeIters; ++it) {
         const uint32_t row = row0 + it * rstep;
         if (row >= n.N) break;
-        const int4 src = srcs[it];
+        int4 src = srcs[it];
+#ifdef WWWS_CHECK_INDICES
+        if (src.x >= 0 && !index_ok(n, src.x, n.N, 103)) src.x = -1;
+        if (src.y >= 0 && !index_ok(n, src.y, n.N, 103)) src.y = -1;
+        if (src.z >= 0 && !index_ok(n, src.z, n.N, 103)) src.z = -1;
+        if (src.w >= 0 && !index_ok(n, src.w, n.N, 103)) src.w = -1;
+#endif
         Q4 acc = ld32(in + uint64_t(row) * ld8);
         Q4 v0, v1, v2, v3;
         if (src.x >= 0) v0 = ld32(in + uint64_t(uint32_t(src.x)) * ld8);
@@ -145,7 +154,9 @@ __global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Ne
         if (src.w >= 0) join(acc, v3);
         if (PUSH) {
             const int32_t* who = n.pullers + rbase * 4 + ins[it].x;
-            for (uint32_t j = 0; j < ins[it].y; ++j) join(acc, ld32(in + uint64_t(uint32_t(who[j])) * ld8));
+            if (index_ok(n, uint64_t(ins[it].x) + ins[it].y, 4ull * n.N + 1, 104))
+                for (uint32_t j = 0; j < ins[it].y; ++j)
+                    if (index_ok(n, uint32_t(who[j]), n.N, 105)) join(acc, ld32(in + uint64_t(uint32_t(who[j])) * ld8));
         }
         st32_stream(out + uint64_t(row) * ld8, acc);
     }
@@ -154,6 +165,7 @@ __global__ void __launch_bounds__(kMergeThreads, PUSH ? 6 : 8) k_gossip_merge(Ne
 // Reverse lists for the pairwise exchange: who pulled each node this round.
 __global__ void k_gossip_indeg(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n.N) return;
     const size_t x = size_t(r) * n.N + i;
@@ -162,12 +174,13 @@ __global__ void k_gossip_indeg(Net n)
     const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
 #pragma unroll
     for (int s = 0; s < 4; ++s)
-        if (p[s] >= 0) atomicAdd(&n.in_deg[size_t(r) * n.N + p[s]], 1u);
+        if (p[s] >= 0 && index_ok(n, p[s], n.N, 106)) atomicAdd(&n.in_deg[size_t(r) * n.N + p[s]], 1u);
 }
 
 // Exclusive prefix sum of the in-degrees of one replica (one block per replica).
 __global__ void __launch_bounds__(1024) k_gossip_scan(Net n)
 {
+    grid_dependency_enter();
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry;
     const uint32_t r = blockIdx.x, lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -198,6 +211,7 @@ __global__ void __launch_bounds__(1024) k_gossip_scan(Net n)
 
 __global__ void k_gossip_fill(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n.N) return;
     const size_t x = size_t(r) * n.N + i;
@@ -206,10 +220,10 @@ __global__ void k_gossip_fill(Net n)
     const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        if (p[s] < 0) continue;
+        if (p[s] < 0 || !index_ok(n, p[s], n.N, 107)) continue;
         const size_t px = size_t(r) * n.N + p[s];
         const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
-        n.pullers[size_t(r) * n.N * 4 + n.in_off[px] + k] = int32_t(i);
+        if (index_ok(n, uint64_t(n.in_off[px]) + k, 4ull * n.N, 108)) n.pullers[size_t(r) * n.N * 4 + n.in_off[px] + k] = int32_t(i);
     }
 }
 
@@ -218,6 +232,7 @@ __global__ void k_gossip_fill(Net n)
 // the puller's entry to the partner.
 __global__ void k_gossip_fixup(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n.N) return;
     const size_t x = size_t(r) * n.N + i;
@@ -235,8 +250,8 @@ __global__ void k_gossip_fixup(Net n)
         if (p[s] == -1) continue;
         if (p[s] < -1) {                             // chosen but dead: the pull failed
             const uint32_t dead = uint32_t(-2 - p[s]);
-            atomicMax(vn + x * n.ld + dead, n.view[x * n.ld + dead] | kOffBit); ++marks;
-        } else atomicMax(vn + (size_t(r) * n.N + p[s]) * n.ld + i, self);
+            if (index_ok(n, dead, n.N, 109)) { atomicMax(vn + x * n.ld + dead, n.view[x * n.ld + dead] | kOffBit); ++marks; }
+        } else if (index_ok(n, p[s], n.N, 110)) atomicMax(vn + (size_t(r) * n.N + p[s]) * n.ld + i, self);
     }
     if (marks) atomicAdd(&n.stats[size_t(r) * sCount + sOfflineMarks], (unsigned long long)marks);
 }
@@ -246,7 +261,7 @@ __global__ void k_gossip_fixup(Net n)
 void launch_scan_in_degrees(const Net& n, const LaunchCtx& c, int kernel_id)
 {
     Timed t(c, kernel_id);
-    k_gossip_scan<<<n.Rp, 1024, 0, c.stream>>>(n);
+    launch_kernel(c, k_gossip_scan, n.Rp, 1024, n);
 }
 
 // Panel width: the widest power of two (32 .. 512 columns) whose panel of N rows fits the
@@ -266,8 +281,8 @@ static uint32_t panel_columns(const Net& n)
 void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c)
 {
     const dim3 pg((n.N + 127) / 128, n.Rp);
-    { Timed t(c, kGossipPeer); k_gossip_peer<<<pg, 128, 0, c.stream>>>(n, round); }
-    { Timed t(c, kGossipPeer); k_gossip_resolve<<<pg, 128, 0, c.stream>>>(n); }
+    { Timed t(c, kGossipPeer); launch_kernel(c, k_gossip_peer, pg, 128, n, round); }
+    { Timed t(c, kGossipPeer); launch_kernel(c, k_gossip_resolve, pg, 128, n); }
     const uint32_t pc = panel_columns(n);
     uint32_t shift = 0;
     while ((4u << shift) < pc) ++shift;                                   // 32-byte chunks per row segment = pc / 4
@@ -276,16 +291,16 @@ void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c)
     const uint32_t groups = (n.N + rows_per_block - 1) / rows_per_block;
     const uint64_t blocks = uint64_t(n.Rp) * n_panels * groups;
     if (n.flags & 8u) {
-        { Timed t(c, kGossipLists); k_gossip_indeg<<<pg, 128, 0, c.stream>>>(n); }
-        { Timed t(c, kGossipLists); k_gossip_scan<<<n.Rp, 1024, 0, c.stream>>>(n); }
-        { Timed t(c, kGossipLists); k_gossip_fill<<<pg, 128, 0, c.stream>>>(n); }
+        { Timed t(c, kGossipLists); launch_kernel(c, k_gossip_indeg, pg, 128, n); }
+        { Timed t(c, kGossipLists); launch_kernel(c, k_gossip_scan, n.Rp, 1024, n); }
+        { Timed t(c, kGossipLists); launch_kernel(c, k_gossip_fill, pg, 128, n); }
         Timed t(c, kGossipMerge);
-        k_gossip_merge<true><<<uint32_t(blocks), kMergeThreads, 0, c.stream>>>(n, pc, shift, n_panels, groups);
+        launch_kernel(c, k_gossip_merge<true>, uint32_t(blocks), kMergeThreads, n, pc, shift, n_panels, groups);
     } else {
         Timed t(c, kGossipMerge);
-        k_gossip_merge<false><<<uint32_t(blocks), kMergeThreads, 0, c.stream>>>(n, pc, shift, n_panels, groups);
+        launch_kernel(c, k_gossip_merge<false>, uint32_t(blocks), kMergeThreads, n, pc, shift, n_panels, groups);
     }
-    { Timed t(c, kGossipFixup); k_gossip_fixup<<<pg, 128, 0, c.stream>>>(n); }
+    { Timed t(c, kGossipFixup); launch_kernel(c, k_gossip_fixup, pg, 128, n); }
 }
 
 }  // namespace wwws

@@ -144,6 +144,7 @@ __device__ __forceinline__ int draw_lanes(const Net& n, Lanes<L>& w, uint32_t q,
 template <int L>
 __global__ void __launch_bounds__(128) k_step_lanes(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     constexpr int RPB = 128 / L;                       // requests per block
     __shared__ BlockStats bs;
     stats_begin(bs);                                   // barrier inside
@@ -243,8 +244,8 @@ int step_lanes_for(uint64_t total)
 void launch_step_lanes(const Net& n, uint64_t first, uint32_t count, int lanes, const LaunchCtx& c)
 {
     Timed t(c, kStepFused);
-    if (lanes == 8) k_step_lanes<8><<<dim3((count + 15) / 16, n.Rp), 128, 0, c.stream>>>(n, first, count);
-    else k_step_lanes<4><<<dim3((count + 31) / 32, n.Rp), 128, 0, c.stream>>>(n, first, count);
+    if (lanes == 8) launch_kernel(c, k_step_lanes<8>, dim3((count + 15) / 16, n.Rp), 128, n, first, count);
+    else launch_kernel(c, k_step_lanes<4>, dim3((count + 31) / 32, n.Rp), 128, n, first, count);
 }
 
 }  // namespace wwws

@@ -17,6 +17,7 @@ __device__ __forceinline__ float ledger_weight(const Net& n, int64_t stake, uint
 __global__ void k_peer_init(Net n, const int64_t* __restrict__ credit0, const uint8_t* __restrict__ online0,
                             uint32_t init_stale_max)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n.N) return;
     const size_t x = size_t(r) * n.N + j;
@@ -39,6 +40,7 @@ __global__ void k_peer_init(Net n, const int64_t* __restrict__ credit0, const ui
 // V[i][j] = entry of j at a version 0..init_stale_max old (own entry current).
 __global__ void k_view_init(Net n, uint32_t init_stale_max)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.z, i = blockIdx.y;
     const uint32_t rg = r + n.replica_offset;
     uint64_t* row = n.view + (size_t(r) * n.N + i) * n.ld;
@@ -56,6 +58,7 @@ __global__ void k_view_init(Net n, uint32_t init_stale_max)
 
 __global__ void k_advance(Net n, uint32_t dt_ms, uint32_t now_ms)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n.N) return;
     const size_t x = size_t(r) * n.N + j;
@@ -92,6 +95,7 @@ __device__ void finalize_replica(const Net& n, uint32_t r)
 // Majority validation: how many peers of each replica are online to confirm a proposed block.
 __global__ void k_count_online(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t on = j < n.N && n.online[size_t(r) * n.N + j];
     const uint32_t c = __reduce_add_sync(0xffffffffu, on);
@@ -100,6 +104,7 @@ __global__ void k_count_online(Net n)
 
 __global__ void k_fold(Net n, int finalize_requested)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     // with majority validation the block is committed only if more than half of the peers are online
     const bool finalize = finalize_requested && (!(n.flags & 32u) || 2u * n.online_count[r] > n.N);
@@ -154,6 +159,7 @@ __global__ void k_fold(Net n, int finalize_requested)
 // The online counts are consumed by one k_fold; clear them for the next proposal.
 __global__ void k_clear_online_count(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r < n.Rp) n.online_count[r] = 0;
 }
@@ -161,6 +167,7 @@ __global__ void k_clear_online_count(Net n)
 // Re-derive stake and weight from the ledger as it stands (after a table import).
 __global__ void k_rederive(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n.N) return;
     const size_t x = size_t(r) * n.N + j;
@@ -174,6 +181,7 @@ __global__ void k_rederive(Net n)
 // credit_total per replica = sum of finalized and pending credit.
 __global__ void k_credit_total(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
     long long s = 0;
     if (j < n.N) { const size_t x = size_t(r) * n.N + j; s = n.credit[x] + n.d_credit[x]; }
@@ -183,6 +191,7 @@ __global__ void k_credit_total(Net n)
 
 __global__ void k_zero_credit_total(Net n)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r < n.Rp) n.stats[size_t(r) * sCount + sCreditTotal] = 0;
 }
@@ -191,36 +200,36 @@ static dim3 peer_grid(const Net& n) { return dim3((n.N + 255) / 256, n.Rp); }
 
 void launch_peer_init(const Net& n, const int64_t* credit0, const uint8_t* online0, uint32_t init_stale_max, const LaunchCtx& c)
 {
-    { Timed t(c, kPeerInit); k_peer_init<<<peer_grid(n), 256, 0, c.stream>>>(n, credit0, online0, init_stale_max); }
+    { Timed t(c, kPeerInit); launch_kernel(c, k_peer_init, peer_grid(n), 256, n, credit0, online0, init_stale_max); }
     const uint32_t bx = (n.ld + 255) / 256 > 64 ? 64 : (n.ld + 255) / 256;
     // grid.y / grid.z limits (65535): rows go in y, replicas in z
-    { Timed t(c, kViewInit); k_view_init<<<dim3(bx, n.N, n.Rp), 256, 0, c.stream>>>(n, init_stale_max); }
+    { Timed t(c, kViewInit); launch_kernel(c, k_view_init, dim3(bx, n.N, n.Rp), 256, n, init_stale_max); }
 }
 
 void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c)
 {
     Timed t(c, kAdvance);
-    k_advance<<<peer_grid(n), 256, 0, c.stream>>>(n, dt_ms, now_ms);
+    launch_kernel(c, k_advance, peer_grid(n), 256, n, dt_ms, now_ms);
 }
 
 void launch_fold(const Net& n, int finalize, const LaunchCtx& c)
 {
     const bool majority = finalize && (n.flags & 32u);
-    if (majority) { Timed t(c, kFold); k_count_online<<<peer_grid(n), 256, 0, c.stream>>>(n); }
-    { Timed t(c, kFold); k_fold<<<peer_grid(n), 256, 0, c.stream>>>(n, finalize); }
-    if (majority) { Timed t(c, kFold); k_clear_online_count<<<(n.Rp + 127) / 128, 128, 0, c.stream>>>(n); }
+    if (majority) { Timed t(c, kFold); launch_kernel(c, k_count_online, peer_grid(n), 256, n); }
+    { Timed t(c, kFold); launch_kernel(c, k_fold, peer_grid(n), 256, n, finalize); }
+    if (majority) { Timed t(c, kFold); launch_kernel(c, k_clear_online_count, (n.Rp + 127) / 128, 128, n); }
 }
 
 void launch_rederive(const Net& n, const LaunchCtx& c)
 {
     Timed t(c, kRederive);
-    k_rederive<<<peer_grid(n), 256, 0, c.stream>>>(n);
+    launch_kernel(c, k_rederive, peer_grid(n), 256, n);
 }
 
 void launch_credit_total(const Net& n, const LaunchCtx& c)
 {
-    { Timed t(c, kCreditTotal); k_zero_credit_total<<<(n.Rp + 127) / 128, 128, 0, c.stream>>>(n); }
-    { Timed t(c, kCreditTotal); k_credit_total<<<peer_grid(n), 256, 0, c.stream>>>(n); }
+    { Timed t(c, kCreditTotal); launch_kernel(c, k_zero_credit_total, (n.Rp + 127) / 128, 128, n); }
+    { Timed t(c, kCreditTotal); launch_kernel(c, k_credit_total, peer_grid(n), 256, n); }
 }
 
 // ---- optional per-kernel event timing ------------------------------------------------------------

@@ -118,6 +118,7 @@ __device__ __forceinline__ uint2 pack_cont(const Window& w, uint32_t mask) { ret
 // Dispatch (D1..D6) of requests [first, first+count) of every replica.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_dispatch(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     __shared__ BlockStats bs;
     stats_begin(bs);
     const uint32_t lane = threadIdx.x & 31, r = blockIdx.y;
@@ -158,6 +159,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_dispatch(Net n, uint64_
 // Duel-and-judge (J1..J3) for the batch last dispatched.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_duel(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     __shared__ BlockStats bs;
     stats_begin(bs);
     const uint32_t lane = threadIdx.x & 31, r = blockIdx.y;
@@ -166,7 +168,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_duel(Net n, uint64_t fi
         const uint64_t q = first + idx;
         const size_t x = size_t(r) * n.Q + q;
         const int a = n.exec_a[x];
-        if (a >= 0) {
+        if (a >= 0 && index_ok(n, a, n.N, 206)) {
             Window w;
             w.r = r; w.rg = r + n.replica_offset; w.q = uint32_t(q); w.o = n.origin[x];
             const Rnd4 rx = draw(n, w.q, 0, w.rg, kOrigin);
@@ -197,6 +199,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32) k_duel(Net n, uint64_t fi
 // Settlement (S1..S4) of the batch, one thread per request.
 __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     __shared__ BlockStats bs;
     stats_begin(bs);
     const uint32_t r = blockIdx.y, idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -217,12 +220,14 @@ __global__ void __launch_bounds__(256) k_settle(Net n, uint64_t first, uint32_t 
 // Scatter the batch's work items into per-peer lists (offsets from the scan of in_deg).
 __global__ void k_fifo_fill(Net n, uint32_t count)
 {
+    grid_dependency_enter();
     const uint32_t r = blockIdx.y, slot = blockIdx.x * blockDim.x + threadIdx.x;
     if (slot >= count * 7) return;
     const int2 item = n.fifo_items[size_t(r) * n.max_batch * 7 + slot];
-    if (item.x < 0) return;
+    if (item.x < 0 || !index_ok(n, item.x, n.N, 201)) return;
     const size_t px = size_t(r) * n.N + item.x;
     const uint32_t k = atomicAdd(&n.in_cursor[px], 1u);
+    if (!index_ok(n, uint64_t(n.in_off[px]) + k, 7ull * n.max_batch, 202)) return;
     // entry: (request, amount): tokens of queued work, or, with bit 31 set, the number of payments of R (role 6)
     n.fifo_list[size_t(r) * n.max_batch * 7 + n.in_off[px] + k] = make_uint2(slot / 7, uint32_t(item.y) | (slot % 7 == 6 ? 0x80000000u : 0u));
 }
@@ -231,6 +236,7 @@ __global__ void k_fifo_fill(Net n, uint32_t count)
 // behind the items that earlier requests of the batch put there.
 __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     __shared__ BlockStats bs;
     stats_begin(bs);
     const uint32_t r = blockIdx.y, idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -239,11 +245,11 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
     if (idx < count) {
         const size_t x = size_t(r) * n.Q + first + idx;
         const int a = n.exec_a[x];
-        if (a != -3 && a != -4) {
+        if (a != -3 && a != -4 && index_ok(n, a < 0 ? n.origin[x] : uint32_t(a), n.N, 203)) {
             const uint32_t ex = a < 0 ? n.origin[x] : uint32_t(a);
             const size_t px = size_t(r) * n.N + ex;
             const uint2* list = n.fifo_list + size_t(r) * n.max_batch * 7 + n.in_off[px];
-            const uint32_t len = n.in_deg[px];
+            const uint32_t len = index_ok(n, uint64_t(n.in_off[px]) + n.in_deg[px], 7ull * n.max_batch + 1, 204) ? n.in_deg[px] : 0u;
             uint64_t ahead = 0;
             for (uint32_t j = 0; j < len; ++j) { const uint2 it = list[j]; if (it.x < idx && !(it.y >> 31)) ahead += it.y; }
             if (a >= 0) {
@@ -251,7 +257,7 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
                 // payer already spent in this block (earlier batches, earlier requests of this batch)
                 const size_t ox = size_t(r) * n.N + n.origin[x];
                 const uint2* mine = n.fifo_list + size_t(r) * n.max_batch * 7 + n.in_off[ox];
-                const uint32_t mlen = n.in_deg[ox];
+                const uint32_t mlen = index_ok(n, uint64_t(n.in_off[ox]) + n.in_deg[ox], 7ull * n.max_batch + 1, 205) ? n.in_deg[ox] : 0u;
                 long long spent = n.blk_spent[ox];
                 for (uint32_t j = 0; j < mlen; ++j) { const uint2 it = mine[j]; if (it.x < idx && (it.y >> 31)) spent += n.R * (long long)(it.y & 0x7fffffffu); }
                 const uint32_t oc = n.outcome[x];
@@ -275,8 +281,8 @@ __global__ void __launch_bounds__(256) k_fifo_latency(Net n, uint64_t first, uin
 void launch_fifo(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
     launch_scan_in_degrees(n, c, kFifo);
-    { Timed t(c, kFifo); k_fifo_fill<<<dim3((count * 7 + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, count); }
-    { Timed t(c, kFifo); k_fifo_latency<<<dim3((count + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, first, count); }
+    { Timed t(c, kFifo); launch_kernel(c, k_fifo_fill, dim3((count * 7 + 255) / 256, n.Rp), 256, n, count); }
+    { Timed t(c, kFifo); launch_kernel(c, k_fifo_latency, dim3((count + 255) / 256, n.Rp), 256, n, first, count); }
 }
 
 static dim3 warp_grid(const Net& n, uint32_t count) { return dim3((count + kWarpsPerBlock - 1) / kWarpsPerBlock, n.Rp); }
@@ -284,16 +290,16 @@ static dim3 warp_grid(const Net& n, uint32_t count) { return dim3((count + kWarp
 void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
     Timed t(c, kDispatch);
-    k_dispatch<<<warp_grid(n, count), kWarpsPerBlock * 32, 0, c.stream>>>(n, first, count);
+    launch_kernel(c, k_dispatch, warp_grid(n, count), kWarpsPerBlock * 32, n, first, count);
 }
 void launch_duel(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
     Timed t(c, kDuel);
-    k_duel<<<warp_grid(n, count), kWarpsPerBlock * 32, 0, c.stream>>>(n, first, count);
+    launch_kernel(c, k_duel, warp_grid(n, count), kWarpsPerBlock * 32, n, first, count);
 }
 void launch_settle(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)
 {
     Timed t(c, kSettle);
-    k_settle<<<dim3((count + 255) / 256, n.Rp), 256, 0, c.stream>>>(n, first, count);
+    launch_kernel(c, k_settle, dim3((count + 255) / 256, n.Rp), 256, n, first, count);
 }
 }  // namespace wwws

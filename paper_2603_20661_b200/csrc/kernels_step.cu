@@ -135,6 +135,7 @@ enum : int { kModeFused = 0, kModeDispatch = 1, kModeDuel = 2 };
 template <int BT, int MODE>
 __global__ void __launch_bounds__(BT, BT == 128 ? kStepBlocksPerSM : 1) k_step_fused(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     __shared__ StepShared<BT> sh;
     stats_begin(sh.stats);                       // barrier inside
     if (threadIdx.x == 0) sh.n_duel = 0;
@@ -173,7 +174,7 @@ __global__ void __launch_bounds__(BT, BT == 128 ? kStepBlocksPerSM : 1) k_step_f
                 } else {
                     // ---- duel call: requests flagged as duels re-create their window and queue up
                     const int a0 = n.exec_a[x];
-                    if (a0 >= 0 && ppm(rx.w[1]) < n.p_duel) {
+                    if (a0 >= 0 && index_ok(n, a0, n.N, 301) && ppm(rx.w[1]) < n.p_duel) {
                         const uint2 ct = n.cont[size_t(r) * n.max_batch + idx];
                         blk = pick_block(n, n.origin[x], rx.w[2]);
                         score_window<BT>(n, sh, slot, r, n.origin[x], blk, ct.x, d);
@@ -297,9 +298,9 @@ static void launch_by_size(const Net& n, uint64_t first, uint32_t count, const L
 {
     // small batches: small blocks, so that the requests spread over all SMs
     if (uint64_t(count) * n.Rp >= 148ull * 128 * 4)
-        k_step_fused<128, MODE><<<dim3((count + 127) / 128, n.Rp), 128, 0, c.stream>>>(n, first, count);
+        launch_kernel(c, k_step_fused<128, MODE>, dim3((count + 127) / 128, n.Rp), 128, n, first, count);
     else
-        k_step_fused<32, MODE><<<dim3((count + 31) / 32, n.Rp), 32, 0, c.stream>>>(n, first, count);
+        launch_kernel(c, k_step_fused<32, MODE>, dim3((count + 31) / 32, n.Rp), 32, n, first, count);
 }
 
 void launch_step_fused(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c, int step_kernel, uint32_t stream_run)

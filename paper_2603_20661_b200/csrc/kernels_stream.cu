@@ -116,18 +116,23 @@ __device__ __forceinline__ void phase_origin(const Net& n, WarpPool& p, Warp& w)
 
 // ---- score: D4 ------------------------------------------------------------------------------------
 // fp32 score of one candidate (0 when it is not eligible or its integer weight truncates to 0),
-// branch-free.  Same IEEE operations, in the same order, as candidate_weight(); an entry that was
-// never heard of (0) and a padding column have advertised capacity 0 and fail that test.
-__device__ __forceinline__ float candidate_score(const Net& n, bool not_self, uint32_t elo, uint32_t ehi, float wl)
+// branch-free.  Same IEEE operations, in the same order, as candidate_weight().  Eligibility by
+// the entry is one range test on its bits 20..39 (advertised capacity and offline bit): capacity
+// in 1..2^19-1 and offline bit clear  <=>  (bits - 1) < 2^19 - 1; an entry that was never heard
+// of (0) and a padding column have capacity 0.  A ledger weight is never negative, so a score of
+// at least 2^-8 (integer weight >= 1) implies a positive weight.  The origin itself is taken out
+// of its own window by the caller.
+template <bool LOAD>
+__device__ __forceinline__ float candidate_score(const Net& n, uint32_t elo, uint32_t ehi, float wl)
 {
-    const uint32_t advcap = __funnelshift_r(elo, ehi, 20) & kCapMax;
+    const uint32_t t = __funnelshift_r(elo, ehi, 20);
     float spare = 1.0f;
-    if (n.flags & 2u) {
-        const float utilf = __fdiv_rn(__uint2float_rn((elo & kQMax) << 4), __fmul_rn(__uint2float_rn(advcap), n.uwf));
-        spare = fmaxf(__fsub_rn(1.0f, utilf), 0.0f);                 // a NaN (0/0 cannot occur: capacity 0 is excluded below) gives 0
+    if (LOAD) {
+        const float utilf = __fdiv_rn(__uint2float_rn((elo & kQMax) << 4), __fmul_rn(__uint2float_rn(t & kCapMax), n.uwf));
+        spare = fmaxf(__fsub_rn(1.0f, utilf), 0.0f);                 // capacity 0 gives inf or NaN here, and 0 after the max
     }
     const float sc = __fmul_rn(wl, spare);
-    const bool ok = not_self && advcap != 0u && !(ehi & 0x80u) && wl > 0.0f && sc >= 0.00390625f;   // weight trunc(256 sc) >= 1
+    const bool ok = ((t & 0xfffffu) - 1u) < kCapMax && sc >= 0.00390625f;
     return ok ? sc : 0.0f;
 }
 
@@ -137,13 +142,14 @@ __device__ __forceinline__ unsigned long long weight_q(float sc)
     return __float2ull_rz(fminf(__fmul_rn(sc, 256.0f), 72057594037927936.0f));
 }
 
-template <bool SCORES>
+template <bool SCORES, bool LOAD>
 __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, uint32_t m)
 {
     const bool active = w.lane < m;
     if (active) {
         const uint2 e = p.q_score[(w.sc_head + w.lane) & (kQ - 1)];
-        const uint32_t slot = p.free_slots[w.n_free - 1u - w.lane];
+        uint32_t slot = p.free_slots[w.n_free - 1u - w.lane];
+        if (!index_ok(n, slot, kSlots, 503)) slot = 0;
         const uint32_t o = e.y & 0xffffu, blk = (e.y >> 16) & 0x7ffu;
         const char* row = reinterpret_cast<const char*>(n.view + (w.pbase + o) * n.ld + kWin * blk);
         const float4* wl4 = reinterpret_cast<const float4*>(n.w_led + size_t(w.r) * n.ld + kWin * blk);
@@ -165,13 +171,20 @@ __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, 
                     const int k = 8 * g2 + j;
                     const uint32_t c = 16u * h + k;
                     const float wl = (k & 3) == 0 ? f[k >> 2].x : (k & 3) == 1 ? f[k >> 2].y : (k & 3) == 2 ? f[k >> 2].z : f[k >> 2].w;
-                    const float sc = candidate_score(n, self != c, v[k >> 2].lo[k & 3], v[k >> 2].hi[k & 3], wl);
+                    float sc = candidate_score<LOAD>(n, v[k >> 2].lo[k & 3], v[k >> 2].hi[k & 3], wl);
+                    if (SCORES) sc = self != c ? sc : 0.0f;            // the checked sum leaves the origin out as it goes
                     p.S[c][slot] = sc;
                     gsum += weight_q(sc);
                     if (SCORES) ssum = __fadd_rn(ssum, sc);
                 }
                 p.G[2 * h + g2][slot] = gsum;
             }
+        }
+        if (!SCORES && self < 32u) {
+            // the origin is not a candidate of its own request: take it out of its window
+            const unsigned long long ws = weight_q(p.S[self][slot]);
+            p.S[self][slot] = 0.0f;
+            p.G[self >> 3][slot] -= ws;
         }
         p.ident[slot] = e.x; p.where[slot] = e.y; p.meta[slot] = 0u; p.picks[slot] = 0u;
         if (SCORES && n.score_sum) n.score_sum[w.xbase + e.x] = ssum;
@@ -192,6 +205,7 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
     uint4 fin = make_uint4(0, 0, 0, 0);
     if (active) {
         slot = p.q_draw[(w.dr_head + w.lane) & (kSlots - 1)];
+        if (!index_ok(n, slot, kSlots, 501)) slot = 0;
         const uint32_t meta = p.meta[slot], where = p.where[slot], idx = p.ident[slot];
         uint32_t picks = p.picks[slot];
         uint32_t n_draws = meta & 0xffu, n_probes = (meta >> 8) & 0xffu, stage = (meta >> 16) & 3u, nj = (meta >> 18) & 7u;
@@ -251,6 +265,7 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
                 p.G[g][slot] = (g == 0 ? G0 : g == 1 ? G1 : g == 2 ? G2 : G3) - wp;
             }
         }
+        if (pick >= 0 && !index_ok(n, kWin * blk + uint32_t(pick), n.N, 502)) pick = -1;
         kind = kCont;
         if (pick < 0) kind = stage == 0 ? kFinNone : (stage == 2 && nj ? kVote : kFinCancel);
         else if (stage < 2) {
@@ -299,7 +314,8 @@ __device__ __forceinline__ void phase_vote(const Net& n, WarpPool& p, Warp& w, u
 {
     const bool active = w.lane < m;
     if (active) {
-        const uint32_t slot = p.q_vote[(w.vo_head + w.lane) & (kSlots - 1)];
+        uint32_t slot = p.q_vote[(w.vo_head + w.lane) & (kSlots - 1)];
+        if (!index_ok(n, slot, kSlots, 504)) slot = 0;
         const uint32_t meta = p.meta[slot], where = p.where[slot], idx = p.ident[slot], picks = p.picks[slot];
         const uint32_t blk = (where >> 16) & 0x7ffu, o = where & 0xffffu, q = uint32_t(w.first + idx);
         const uint32_t nj = (meta >> 18) & 7u;
@@ -351,9 +367,10 @@ __device__ __forceinline__ void phase_finish(const Net& n, WarpPool& p, Warp& w,
 
 enum : int { phOrigin, phScore, phDraw, phVote, phFinish, phDone };
 
-template <bool GREEDY, bool SCORES>
+template <bool GREEDY, bool SCORES, bool LOAD>
 __global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, uint32_t count)
 {
+    grid_dependency_enter();
     __shared__ WarpPool p;
     Warp w;
     w.lane = threadIdx.x; w.lt = (1u << w.lane) - 1u;
@@ -395,7 +412,7 @@ __global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, u
         __syncwarp();
         switch (ph) {
         case phOrigin: phase_origin<SCORES>(n, p, w); break;
-        case phScore: phase_score<SCORES>(n, p, w, m); break;
+        case phScore: phase_score<SCORES, LOAD>(n, p, w, m); break;
         case phDraw: phase_draw<GREEDY, SCORES>(n, p, w, m); break;
         case phVote: phase_vote(n, p, w, m, acc); break;
         default: phase_finish(n, p, w, m, acc); break;
@@ -430,18 +447,30 @@ static uint32_t stream_warps_per_replica(const Net& n, uint32_t count, uint32_t 
     return g > chunks ? chunks : g;
 }
 
-template <bool GREEDY, bool SCORES>
+template <bool GREEDY, bool SCORES, bool LOAD>
 static void launch_stream_variant(const Net& n, uint64_t first, uint32_t count, uint32_t run, const LaunchCtx& c)
 {
     static const int resident = [] {
         int dev = 0, sms = 0, per_sm = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_step_stream<GREEDY, SCORES>, 32, 0);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_step_stream<GREEDY, SCORES, LOAD>, 32, 0);
         return sms * per_sm > 0 ? sms * per_sm : 148 * 15;
     }();
     const dim3 grid(stream_warps_per_replica(n, count, run, resident), n.Rp);
-    k_step_stream<GREEDY, SCORES><<<grid, 32, 0, c.stream>>>(n, first, count);
+    // A plain stream-ordered launch: this kernel wants the SM's whole shared memory, and blocks that
+    // arrive while the previous kernel's blocks still hold the SM in another shared-memory
+    // configuration get a fraction of the occupancy for their whole (long) life.
+    LaunchCtx plain = c;
+    plain.overlap = false;
+    launch_kernel(plain, k_step_stream<GREEDY, SCORES, LOAD>, grid, 32, n, first, count);
+}
+
+template <bool GREEDY, bool SCORES>
+static void launch_stream_load(const Net& n, uint64_t first, uint32_t count, uint32_t run, const LaunchCtx& c)
+{
+    if (n.flags & 2u) launch_stream_variant<GREEDY, SCORES, true>(n, first, count, run, c);
+    else launch_stream_variant<GREEDY, SCORES, false>(n, first, count, run, c);
 }
 
 void launch_step_stream(const Net& n, uint64_t first, uint32_t count, uint32_t run, const LaunchCtx& c)
@@ -449,11 +478,11 @@ void launch_step_stream(const Net& n, uint64_t first, uint32_t count, uint32_t r
     Timed t(c, kStepFused);
     const bool scores = n.score_a || n.score_sum;
     if (n.flags & 4u) {
-        if (scores) launch_stream_variant<true, true>(n, first, count, run, c);
-        else launch_stream_variant<true, false>(n, first, count, run, c);
+        if (scores) launch_stream_load<true, true>(n, first, count, run, c);
+        else launch_stream_load<true, false>(n, first, count, run, c);
     } else {
-        if (scores) launch_stream_variant<false, true>(n, first, count, run, c);
-        else launch_stream_variant<false, false>(n, first, count, run, c);
+        if (scores) launch_stream_load<false, true>(n, first, count, run, c);
+        else launch_stream_load<false, false>(n, first, count, run, c);
     }
 }
 

@@ -84,6 +84,7 @@ __device__ __forceinline__ uint64_t weight_of(float sc)
 __device__ __forceinline__ bool probe_peer(const Net& n, uint32_t r, uint32_t rg, uint32_t q, uint32_t blk, int pick)
 {
     const size_t x = size_t(r) * n.N + kWin * blk + pick;
+    if (!index_ok(n, kWin * blk + uint32_t(pick), n.N, 409)) return false;
     const uint32_t cap = n.cap_eff[x];
     const uint8_t on = n.online[x];
     const int64_t queued = n.backlog[x];
@@ -144,8 +145,9 @@ struct SettleAcc {
 // k_fifo_latency computes the latencies once the per-peer lists are built.
 __device__ __forceinline__ void fifo_emit(const Net& n, uint32_t r, uint32_t bidx, uint32_t role, int peer, uint32_t tokens)
 {
+    if (!index_ok(n, bidx, n.max_batch, 407)) return;
     n.fifo_items[(size_t(r) * n.max_batch + bidx) * 7 + role] = make_int2(peer, int(tokens));
-    if (peer >= 0) atomicAdd(&n.in_deg[size_t(r) * n.N + peer], 1u);
+    if (peer >= 0 && index_ok(n, uint32_t(peer), n.N, 408)) atomicAdd(&n.in_deg[size_t(r) * n.N + peer], 1u);
 }
 
 // S3 of a decided duel (outcome 1..3): the challenger's execution and payment, the judges' work,
@@ -158,6 +160,13 @@ __device__ __forceinline__ long long settle_duel(const Net& n, uint32_t r, uint3
     const size_t base = size_t(r) * n.N;
     const uint64_t key = chain_key(n, r);
     const uint64_t work = uint64_t(li) + lo;
+#ifdef WWWS_CHECK_INDICES
+    {
+        bool ok = index_ok(n, uint32_t(a), n.N, 401) && index_ok(n, uint32_t(b), n.N, 402) && index_ok(n, o, n.N, 403);
+        for (int l = 0; l < 4; ++l) if (jd[l] >= 0) ok = ok && index_ok(n, uint32_t(jd[l]), n.N, 404);
+        if (!ok) return 0;
+    }
+#endif
     s.digest += record_hash(key, q, opPayChallenger, o, -n.R) + record_hash(key, q, opEarnChallenger, uint32_t(b), n.R);
     add64(&n.d_credit[base + b], n.R);
     add64(&n.d_backlog[base + b], (long long)work);
@@ -211,6 +220,7 @@ __device__ __forceinline__ void settle_one(const Net& n, uint32_t r, uint32_t q,
     if (near) s.add(sNear);
     if (a == -3) { s.add(sDropped); return; }
     if (a == -4) { s.add(sFailed); return; }
+    if (!index_ok(n, o, n.N, 405) || (a >= 0 && !index_ok(n, uint32_t(a), n.N, 406))) return;
     uint32_t ex;
     if (a < 0) {
         if (a == -1) s.add(sLocal); else s.add(sFallback);

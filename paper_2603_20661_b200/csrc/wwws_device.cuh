@@ -19,7 +19,7 @@ enum : uint32_t { sRequests, sLocal, sFallback, sDropped, sFailed, sDelegated, s
                   sChainHead, sPendingDigest, sUncovered, sBlocksRejected, sCount };
 
 // Device error word codes (subset of wwws_status).
-enum : uint32_t { eArg = 1, eRange = 4, eInvariant = 6 };
+enum : uint32_t { eArg = 1, eRange = 4, eInvariant = 6, eIndex = 8 };
 
 // Everything a kernel needs, passed by value.  Per-peer arrays are [Rp][N]; the view is
 // [Rp][N][ld] with ld = N rounded up to 32 so that a candidate window is one aligned
@@ -74,6 +74,15 @@ struct Net {
     int32_t* exec_a; int32_t* exec_b; int32_t* judges; uint8_t* outcome; uint8_t* rflags;
     float* score_a; float* score_sum;
 };
+
+// First statement of every kernel: let the next grid of the stream be scheduled already, then wait
+// until the previous grid has completed and its memory operations are visible.  Without the
+// programmatic-serialization launch attribute both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_enter()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 
 struct Rnd4 { uint32_t w[4]; };
 
@@ -167,5 +176,20 @@ __device__ __forceinline__ void set_error(const Net& n, uint32_t code, uint32_t 
 {
     if (atomicCAS(&n.err[0], 0u, code) == 0u) n.err[1] = detail;
 }
+
+// Checked build (-DWWWS_CHECK_INDICES): every index that a kernel takes from device data (partner
+// ids, list offsets, candidate and executor ids, queue slots) is range-checked before use; a bad
+// one sets the device error word (code eIndex, detail = the site's tag) and the access is skipped.
+// Nothing traps.  In the normal build the test compiles to `true`.
+#ifdef WWWS_CHECK_INDICES
+__device__ __forceinline__ bool index_ok(const Net& n, uint64_t i, uint64_t limit, uint32_t tag)
+{
+    if (i < limit) return true;
+    set_error(n, eIndex, tag);
+    return false;
+}
+#else
+__device__ __forceinline__ bool index_ok(const Net&, uint64_t, uint64_t, uint32_t) { return true; }
+#endif
 
 }  // namespace wwws

@@ -30,6 +30,7 @@ struct LaunchCtx {
     cudaStream_t stream;
     uint64_t* launches;          // total kernels launched
     Profiler* prof;
+    bool overlap;                // launch with programmatic stream serialization (see launch_kernel)
 };
 
 struct Timed {                   // RAII bracket around one launch
@@ -37,6 +38,23 @@ struct Timed {                   // RAII bracket around one launch
     Timed(const LaunchCtx& ctx, int id) : c(ctx) { *c.launches += 1; if (c.prof && c.prof->enabled) c.prof->begin(id, c.stream); }
     ~Timed() { if (c.prof && c.prof->enabled) c.prof->end(c.stream); }
 };
+
+// Every kernel of the library is launched through here.  With `overlap` the launch carries the
+// programmatic-stream-serialization attribute: the grid may be scheduled while its predecessor in
+// the stream is still running, and its threads hold at grid_dependency_enter() (the first
+// statement of every kernel) until the predecessor has completed and its writes are visible.
+// What overlaps is the launch latency and the block scheduling, not the work.
+template <class... P, class... A>
+inline void launch_kernel(const LaunchCtx& c, void (*kernel)(P...), dim3 grid, dim3 block, A&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = c.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = c.overlap ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
 
 void launch_peer_init(const Net& n, const int64_t* credit0, const uint8_t* online0, uint32_t init_stale_max, const LaunchCtx& c);
 void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c);
