@@ -176,6 +176,8 @@ class Leg:
             self.net.set_option(1, args.step_kernel)
         if args.stream_run:
             self.net.set_option(2, args.stream_run)
+        if args.host_io:
+            self.net.set_option(4, args.host_io)
         if args.overlap is not None:
             self.net.set_option(3, args.overlap)
         self.W, self.s = args.warmup, 0
@@ -531,6 +533,7 @@ def main(argv=None):
     ap.add_argument("--batch", type=int, default=None, help="override requests per replica per step (saturation runs)")
     ap.add_argument("--step-kernel", type=int, default=0, help="force the fused step's kernel (WWWS_OPT_STEP_KERNEL)")
     ap.add_argument("--stream-run", type=int, default=0, help="requests per warp of the streaming kernel (WWWS_OPT_STREAM_RUN)")
+    ap.add_argument("--host-io", type=int, default=0, help="wwws_step_host path: 0 by batch size, 1 mapped direct, 2 staged (WWWS_OPT_HOST_IO)")
     ap.add_argument("--overlap", type=int, default=None, help="mask of launches that may overlap their predecessor (WWWS_OPT_LAUNCH_OVERLAP)")
     ap.add_argument("--sustain-s", type=float, default=1.0, help="device seconds of the repeated timed region")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))

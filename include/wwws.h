@@ -232,7 +232,7 @@ typedef struct {
 /* wwws_step with HOST buffers; synchronises before it returns.  totals_out (HOST, one record) may be NULL.
  * Two ways, with identical results.  Direct: if all eight buffers are page-locked and mapped into the device's
  * address space (cudaHostAlloc, cudaHostRegister), exact queueing (WWWS_FLAG_FIFO) is off and the batch is small
- * (n_replicas * count <= 16384, or WWWS_OPT_HOST_IO = 1), the kernels read the batch's requests from, and write
+ * (n_replicas * count <= 98304, or WWWS_OPT_HOST_IO = 1), the kernels read the batch's requests from, and write
  * its results to, the host buffers themselves; the bound device arrays are not touched.  Staged: the batch's
  * request slices are copied to the bound device arrays on a second stream (created at the first such call)
  * while time advance and gossip run, the step runs on the device arrays, and the batch's results are copied

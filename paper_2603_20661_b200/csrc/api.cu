@@ -29,6 +29,8 @@ struct wwws_network {
     uint64_t launches;
     Profiler prof;
     std::string err;
+    bool fold_pending = false;   // wwws_step left its fold to the next call (see settle_pending)
+    int fold_finalize = 0;
     int host_io = 0;             // wwws_step_host: 0 by batch size, 1 kernels use mapped host buffers, 2 staged copies
     cudaStream_t copy_stream = nullptr;          // staged host path: copies run beside the kernels
     cudaEvent_t ev_fork = nullptr, ev_in = nullptr, ev_step = nullptr;
@@ -174,6 +176,16 @@ wwws_status launch_status(wwws_network* n, const char* what)
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(n, WWWS_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
     return WWWS_OK;
+}
+
+// wwws_step does not fold its batch (queues, block commit) itself: the next wwws_step does it in
+// the same launch as its time advance.  Every other call that reads or changes the state folds
+// first, so the deferral is never visible.
+void settle_pending(wwws_network* n)
+{
+    if (!n->fold_pending) return;
+    n->fold_pending = false;
+    launch_fold(n->d, n->fold_finalize, n->ctx(8));
 }
 
 }  // namespace
@@ -328,6 +340,7 @@ wwws_status wwws_advance_time(wwws_network* n, uint32_t now_ms)
     if (now_ms < n->t_last_ms) return fail(n, WWWS_ERR_ARG, "time must not go back");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "advance_time inside a batch");
     ON_DEVICE(n);
+    settle_pending(n);
     launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx());
     n->t_last_ms = now_ms;
     return launch_status(n, "advance_time");
@@ -338,6 +351,7 @@ wwws_status wwws_gossip_round(wwws_network* n)
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "gossip_round inside a batch");
     ON_DEVICE(n);
+    settle_pending(n);
     launch_gossip(n->d, n->round, n->ctx());
     std::swap(n->d.view, n->d.view_new);
     n->round += 1;
@@ -368,6 +382,7 @@ wwws_status wwws_dispatch_batch(wwws_network* n, uint64_t first, uint64_t count)
 {
     if (wwws_status st = check_batch(n, first, count)) return st;
     ON_DEVICE(n);
+    settle_pending(n);
     if (threads_for(n, count)) launch_dispatch_threads(n->d, first, uint32_t(count), n->ctx());
     else launch_dispatch(n->d, first, uint32_t(count), n->ctx());
     n->batch_first = first; n->batch_count = uint32_t(count); n->phase = 1;
@@ -402,7 +417,13 @@ wwws_status wwws_settle_credits(wwws_network* n, int finalize)
 static wwws_status step_impl(wwws_network* n, uint64_t first, uint64_t count, uint32_t now_ms, int do_gossip, int finalize,
                              cudaEvent_t inputs_ready, cudaEvent_t results_ready)
 {
-    launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx(1));
+    if (n->fold_pending && !(n->d.flags & 32u)) {
+        n->fold_pending = false;
+        launch_fold_advance(n->d, n->fold_finalize, now_ms - n->t_last_ms, now_ms, n->ctx(1));
+    } else {
+        settle_pending(n);
+        launch_advance(n->d, now_ms - n->t_last_ms, now_ms, n->ctx(1));
+    }
     n->t_last_ms = now_ms;
     if (do_gossip) {
         launch_gossip(n->d, n->round, n->ctx(2));
@@ -413,7 +434,8 @@ static wwws_status step_impl(wwws_network* n, uint64_t first, uint64_t count, ui
     launch_step_fused(n->d, first, uint32_t(count), n->ctx(4), n->step_kernel, n->stream_run);
     if (results_ready) CUDA_TRY(n, cudaEventRecord(results_ready, n->stream));
     if (n->d.flags & 16u) launch_fifo(n->d, first, uint32_t(count), n->ctx(4));
-    launch_fold(n->d, finalize != 0, n->ctx(8));
+    n->fold_pending = true;                      // folded by the next call, whichever it is
+    n->fold_finalize = finalize != 0;
     return launch_status(n, "step");
 }
 
@@ -434,47 +456,54 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
     ON_DEVICE(n);
     if (now_ms < n->t_last_ms) return fail(n, WWWS_ERR_ARG, "time must not go back");
     // Large batches go through staged copies even when the buffers are mapped: result records written
-    // across the bus request by request, in the order the kernel finishes them, cost more than three
-    // strided copies that run beside the kernels.
-    const bool want_direct = n->host_io == 1 || (n->host_io == 0 && count * n->d.Rp <= 16384);
-    if (!(n->d.flags & 16u) && want_direct) {
+    // across the bus request by request, in the order the kernel finishes them, cost more than two
+    // small copy kernels that run beside the others (measured per step, direct / staged: 64,000
+    // requests 0.67 / 0.70 ms, 128,000 requests 0.94 / 0.62 ms).
+    const bool want_direct = n->host_io == 1 || (n->host_io == 0 && count * n->d.Rp <= 98304);
+    // are all eight buffers page-locked and mapped into the device's address space?
+    const void* host[8] = { io->origin, io->len_in, io->len_out, io->exec_a, io->exec_b, io->judges, io->outcome, io->flags };
+    void* dev[8];
+    bool mapped = true;
+    for (int k = 0; k < 8 && mapped; ++k) {
+        cudaPointerAttributes a;
+        if (cudaPointerGetAttributes(&a, host[k]) != cudaSuccess) { cudaGetLastError(); mapped = false; }
+        else if (a.type != cudaMemoryTypeHost || !a.devicePointer) mapped = false;
+        else dev[k] = a.devicePointer;
+    }
+    if (mapped && (reinterpret_cast<uintptr_t>(dev[5]) & 15) != 0) mapped = false;
+    HostBatch hb{};
+    if (mapped) {
+        hb.origin = static_cast<const uint32_t*>(dev[0]); hb.len_in = static_cast<const uint16_t*>(dev[1]);
+        hb.len_out = static_cast<const uint16_t*>(dev[2]);
+        hb.exec_a = static_cast<int32_t*>(dev[3]); hb.exec_b = static_cast<int32_t*>(dev[4]); hb.judges = static_cast<int32_t*>(dev[5]);
+        hb.outcome = static_cast<uint8_t*>(dev[6]); hb.rflags = static_cast<uint8_t*>(dev[7]);
+    }
+    if (!(n->d.flags & 16u) && want_direct && mapped) {
         // Page-locked, mapped host buffers are read and written by the kernels themselves: no copies,
         // and the result stores travel while the step runs.  (With exact queueing the results are
         // read again by later kernels, which is better done from device memory.)
-        const void* host[8] = { io->origin, io->len_in, io->len_out, io->exec_a, io->exec_b, io->judges, io->outcome, io->flags };
-        void* dev[8];
-        bool direct = true;
-        for (int k = 0; k < 8 && direct; ++k) {
-            cudaPointerAttributes a;
-            if (cudaPointerGetAttributes(&a, host[k]) != cudaSuccess) { cudaGetLastError(); direct = false; }
-            else if (a.type != cudaMemoryTypeHost || !a.devicePointer) direct = false;
-            else dev[k] = a.devicePointer;
+        Net& d = n->d;
+        const Net saved = d;
+        d.origin = hb.origin; d.len_in = hb.len_in; d.len_out = hb.len_out;
+        d.exec_a = hb.exec_a; d.exec_b = hb.exec_b; d.judges = hb.judges; d.outcome = hb.outcome; d.rflags = hb.rflags;
+        d.score_a = nullptr; d.score_sum = nullptr;
+        const wwws_status st = step_impl(n, first, count, now_ms, do_gossip, finalize, nullptr, nullptr);
+        d.origin = saved.origin; d.len_in = saved.len_in; d.len_out = saved.len_out;
+        d.exec_a = saved.exec_a; d.exec_b = saved.exec_b; d.judges = saved.judges; d.outcome = saved.outcome; d.rflags = saved.rflags;
+        d.score_a = saved.score_a; d.score_sum = saved.score_sum;
+        if (st) return st;
+        if (totals_out) {
+            std::vector<wwws_stats_t> all(d.Rp + 1);
+            if (wwws_status st2 = wwws_stats(n, all.data())) return st2;
+            *totals_out = all[d.Rp];
+            return WWWS_OK;
         }
-        if (direct && (reinterpret_cast<uintptr_t>(dev[5]) & 15) == 0) {
-            Net& d = n->d;
-            const Net saved = d;
-            d.origin = static_cast<const uint32_t*>(dev[0]); d.len_in = static_cast<const uint16_t*>(dev[1]);
-            d.len_out = static_cast<const uint16_t*>(dev[2]);
-            d.exec_a = static_cast<int32_t*>(dev[3]); d.exec_b = static_cast<int32_t*>(dev[4]); d.judges = static_cast<int32_t*>(dev[5]);
-            d.outcome = static_cast<uint8_t*>(dev[6]); d.rflags = static_cast<uint8_t*>(dev[7]);
-            d.score_a = nullptr; d.score_sum = nullptr;
-            const wwws_status st = step_impl(n, first, count, now_ms, do_gossip, finalize, nullptr, nullptr);
-            d.origin = saved.origin; d.len_in = saved.len_in; d.len_out = saved.len_out;
-            d.exec_a = saved.exec_a; d.exec_b = saved.exec_b; d.judges = saved.judges; d.outcome = saved.outcome; d.rflags = saved.rflags;
-            d.score_a = saved.score_a; d.score_sum = saved.score_sum;
-            if (st) return st;
-            if (totals_out) {
-                std::vector<wwws_stats_t> all(d.Rp + 1);
-                if (wwws_status st2 = wwws_stats(n, all.data())) return st2;
-                *totals_out = all[d.Rp];
-                return WWWS_OK;
-            }
-            return check_device_error(n);
-        }
+        return check_device_error(n);
     }
     // Staged path: the batch's request slices go to the bound device arrays on a second stream while
     // time advance and gossip run; the request kernel waits for them; the results travel back on the
-    // second stream while the block is folded and the counters are read.
+    // second stream while the block is folded and the counters are read.  Mapped buffers are moved by
+    // two small kernels (whole 128-byte lines across the bus, in request order), others by strided copies.
     if (!n->copy_stream) {
         CUDA_TRY(n, cudaStreamCreateWithFlags(&n->copy_stream, cudaStreamNonBlocking));
         CUDA_TRY(n, cudaEventCreateWithFlags(&n->ev_fork, cudaEventDisableTiming));
@@ -483,22 +512,30 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
     }
     const Net& d = n->d;
     cudaStream_t cs = n->copy_stream;
+    LaunchCtx cctx = n->ctx(0);
+    cctx.stream = cs;
     const size_t Q = d.Q, Rp = d.Rp, c = count;
     // the batch is one strided slice per array: Rp rows of `count` elements, pitch n_requests
 #define COPY2D(dst, src, T, W, kind) CUDA_TRY(n, cudaMemcpy2DAsync((void*)((dst) + first * (W)), Q * sizeof(T) * (W), (src) + first * (W), Q * sizeof(T) * (W), c * sizeof(T) * (W), Rp, kind, cs))
     CUDA_TRY(n, cudaEventRecord(n->ev_fork, n->stream));               // whatever still reads the device arrays comes first
     CUDA_TRY(n, cudaStreamWaitEvent(cs, n->ev_fork, 0));
-    COPY2D(d.origin, io->origin, uint32_t, 1, cudaMemcpyHostToDevice);
-    COPY2D(d.len_in, io->len_in, uint16_t, 1, cudaMemcpyHostToDevice);
-    COPY2D(d.len_out, io->len_out, uint16_t, 1, cudaMemcpyHostToDevice);
+    if (mapped) launch_host_batch_in(d, hb, first, uint32_t(count), cctx);
+    else {
+        COPY2D(d.origin, io->origin, uint32_t, 1, cudaMemcpyHostToDevice);
+        COPY2D(d.len_in, io->len_in, uint16_t, 1, cudaMemcpyHostToDevice);
+        COPY2D(d.len_out, io->len_out, uint16_t, 1, cudaMemcpyHostToDevice);
+    }
     CUDA_TRY(n, cudaEventRecord(n->ev_in, cs));
     if (wwws_status st = step_impl(n, first, count, now_ms, do_gossip, finalize, n->ev_in, n->ev_step)) { cudaStreamSynchronize(cs); return st; }
     CUDA_TRY(n, cudaStreamWaitEvent(cs, n->ev_step, 0));
-    COPY2D(io->exec_a, d.exec_a, int32_t, 1, cudaMemcpyDeviceToHost);
-    COPY2D(io->exec_b, d.exec_b, int32_t, 1, cudaMemcpyDeviceToHost);
-    COPY2D(io->judges, d.judges, int32_t, 4, cudaMemcpyDeviceToHost);
-    COPY2D(io->outcome, d.outcome, uint8_t, 1, cudaMemcpyDeviceToHost);
-    COPY2D(io->flags, d.rflags, uint8_t, 1, cudaMemcpyDeviceToHost);
+    if (mapped) launch_host_batch_out(d, hb, first, uint32_t(count), cctx);
+    else {
+        COPY2D(io->exec_a, d.exec_a, int32_t, 1, cudaMemcpyDeviceToHost);
+        COPY2D(io->exec_b, d.exec_b, int32_t, 1, cudaMemcpyDeviceToHost);
+        COPY2D(io->judges, d.judges, int32_t, 4, cudaMemcpyDeviceToHost);
+        COPY2D(io->outcome, d.outcome, uint8_t, 1, cudaMemcpyDeviceToHost);
+        COPY2D(io->flags, d.rflags, uint8_t, 1, cudaMemcpyDeviceToHost);
+    }
 #undef COPY2D
     wwws_status st = WWWS_OK;
     if (totals_out) {
@@ -507,6 +544,7 @@ wwws_status wwws_step_host(wwws_network* n, const wwws_host_io* io, uint64_t fir
         if (!st) *totals_out = all[Rp];
     } else st = check_device_error(n);
     CUDA_TRY(n, cudaStreamSynchronize(cs));
+    if (cudaError_t e = cudaGetLastError(); e != cudaSuccess && !st) return fail(n, WWWS_ERR_CUDA, std::string("step_host copies: ") + cudaGetErrorString(e));
     return st;
 }
 
@@ -515,6 +553,7 @@ wwws_status wwws_stats(wwws_network* n, wwws_stats_t* host_out)
     if (!n) return fail(nullptr, WWWS_ERR_ARG, "network is NULL");
     if (!host_out) return fail(n, WWWS_ERR_ARG, "host_out is NULL");
     ON_DEVICE(n);
+    settle_pending(n);
     launch_credit_total(n->d, n->ctx());
     if (wwws_status st = launch_status(n, "stats")) return st;
     CUDA_TRY(n, cudaMemcpyAsync(host_out, n->d.stats, uint64_t(n->d.Rp) * sizeof(wwws_stats_t), cudaMemcpyDeviceToHost, n->stream));
@@ -535,6 +574,7 @@ wwws_status wwws_export_table(wwws_network* n, wwws_table t, void* host_dst, uin
     const uint64_t need = uint64_t(n->d.N) * n->d.Rp * n->tables[t].elem;
     if (bytes != need) return fail(n, WWWS_ERR_ARG, "bytes does not match the table size");
     ON_DEVICE(n);
+    settle_pending(n);
     CUDA_TRY(n, cudaMemcpyAsync(host_dst, n->tables[t].ptr, need, cudaMemcpyDeviceToHost, n->stream));
     return check_device_error(n);
 }
@@ -547,6 +587,7 @@ wwws_status wwws_import_table(wwws_network* n, wwws_table t, const void* host_sr
     const uint64_t need = uint64_t(n->d.N) * n->d.Rp * n->tables[t].elem;
     if (bytes != need) return fail(n, WWWS_ERR_ARG, "bytes does not match the table size");
     ON_DEVICE(n);
+    settle_pending(n);
     CUDA_TRY(n, cudaMemcpyAsync(n->tables[t].ptr, host_src, need, cudaMemcpyHostToDevice, n->stream));
     if (t == WWWS_T_CREDIT || t == WWWS_T_WINS || t == WWWS_T_DUELS || t == WWWS_T_ONLINE || t == WWWS_T_CAP_EFF || t == WWWS_T_BACKLOG)
         launch_rederive(n->d, n->ctx());           // stakes, ledger weights and the peers' gates follow the tables
@@ -602,6 +643,7 @@ wwws_status wwws_import_stats(wwws_network* n, const wwws_stats_t* host_src)
     if (!host_src) return fail(n, WWWS_ERR_ARG, "host_src is NULL");
     if (n->phase != 0) return fail(n, WWWS_ERR_STATE, "import inside a batch");
     ON_DEVICE(n);
+    settle_pending(n);
     CUDA_TRY(n, cudaMemcpyAsync(n->d.stats, host_src, uint64_t(n->d.Rp) * sizeof(wwws_stats_t), cudaMemcpyHostToDevice, n->stream));
     CUDA_TRY(n, cudaStreamSynchronize(n->stream));
     return WWWS_OK;
@@ -663,7 +705,7 @@ const char* wwws_profile_kernel_name(uint32_t k)
 {
     static const char* names[kKernelCount] = { "k_peer_init", "k_view_init", "k_advance", "k_fold",
         "k_rederive", "k_credit_total", "k_gossip_peer", "k_gossip_merge", "k_gossip_fixup", "k_gossip_lists", "k_fifo", "k_dispatch", "k_duel",
-        "k_settle", "k_step_fused" };
+        "k_settle", "k_step_fused", "k_host_batch" };
     return k < kKernelCount ? names[k] : "";
 }
 
@@ -708,6 +750,7 @@ extern "C" wwws_status wwws_gossip_round_static(wwws_network* n)
     const int dev = n->device;
     if (dev < 0 || dev >= kMaxDevices) return fail(n, WWWS_ERR_ARG, "device ordinal beyond 63");
     ON_DEVICE(n);
+    settle_pending(n);
     void* p = g_gossip_scratch_addr[dev].load(std::memory_order_acquire);
     if (!p) {
         // In host code the array's name is only a handle for the runtime; the address the

@@ -227,9 +227,13 @@ __global__ void k_gossip_fill(Net n)
     }
 }
 
-// The three single-entry updates of a round, all joins (max), applied after the row merge:
-// own fresh entry, offline mark for a partner that did not answer, and the "hello" that shows
-// the puller's entry to the partner.
+// The three single-entry updates of a round, applied after the row merge: own fresh entry,
+// offline mark for a partner that did not answer, and the "hello" that shows the puller's entry
+// to the partner.  None needs an atomic.  A peer that is online has just issued a new version,
+// and nobody else can hold that version yet, so its fresh entry is the maximum wherever it
+// lands: own entry and hellos are plain stores (two pullers of one partner write different
+// columns).  An offline mark is a read-max-write of an element that only this thread writes: a
+// hello into the same element would have to come from the dead partner, which sends none.
 __global__ void k_gossip_fixup(Net n)
 {
     grid_dependency_enter();
@@ -240,8 +244,8 @@ __global__ void k_gossip_fixup(Net n)
     n.in_deg[x] = 0;                                 // the reverse lists of this round are spent
     if (!n.online[x]) return;
     const uint64_t self = n.self_entry[x];
-    unsigned long long* vn = reinterpret_cast<unsigned long long*>(n.view_new);
-    atomicMax(vn + x * n.ld + i, self);
+    uint64_t* vn = n.view_new;
+    vn[x * n.ld + i] = self;
     const int4 p4 = *reinterpret_cast<const int4*>(n.partner + x * 4);
     const int32_t p[4] = { p4.x, p4.y, p4.z, p4.w };
     uint32_t marks = 0;
@@ -250,8 +254,12 @@ __global__ void k_gossip_fixup(Net n)
         if (p[s] == -1) continue;
         if (p[s] < -1) {                             // chosen but dead: the pull failed
             const uint32_t dead = uint32_t(-2 - p[s]);
-            if (index_ok(n, dead, n.N, 109)) { atomicMax(vn + x * n.ld + dead, n.view[x * n.ld + dead] | kOffBit); ++marks; }
-        } else if (index_ok(n, p[s], n.N, 110)) atomicMax(vn + (size_t(r) * n.N + p[s]) * n.ld + i, self);
+            if (index_ok(n, dead, n.N, 109)) {
+                const uint64_t mark = n.view[x * n.ld + dead] | kOffBit, cur = vn[x * n.ld + dead];
+                if (mark > cur) vn[x * n.ld + dead] = mark;
+                ++marks;
+            }
+        } else if (index_ok(n, p[s], n.N, 110)) vn[(size_t(r) * n.N + p[s]) * n.ld + i] = self;
     }
     if (marks) atomicAdd(&n.stats[size_t(r) * sCount + sOfflineMarks], (unsigned long long)marks);
 }

@@ -102,7 +102,10 @@ __global__ void k_count_online(Net n)
     if ((threadIdx.x & 31) == 0 && c) atomicAdd(&n.online_count[r], c);
 }
 
-__global__ void k_fold(Net n, int finalize_requested)
+// ADVANCE: the time advance of the next step in the same pass (the step's fold was deferred to the
+// next step's call): one launch and one sweep over the per-peer tables instead of two.
+template <bool ADVANCE>
+__global__ void k_fold(Net n, int finalize_requested, uint32_t dt_ms, uint32_t now_ms)
 {
     grid_dependency_enter();
     const uint32_t r = blockIdx.y, j = blockIdx.x * blockDim.x + threadIdx.x;
@@ -113,7 +116,7 @@ __global__ void k_fold(Net n, int finalize_requested)
         const size_t x = size_t(r) * n.N + j;
         const long long db = n.d_backlog[x];
         const int64_t queued = n.backlog[x] + db;
-        if (db) { n.backlog[x] = queued; n.d_backlog[x] = 0; }
+        if (db) n.d_backlog[x] = 0;
         int64_t credit_now = n.credit[x];
         if (n.flags & 16u) {
             n.in_deg[x] = 0;                         // per-peer item counts of the batch's queueing pass
@@ -131,7 +134,23 @@ __global__ void k_fold(Net n, int finalize_requested)
             csum = c;
             credit_now = c;
         }
-        if (db || finalize) refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], queued, credit_now);
+        if (ADVANCE) {
+            // C3 on top of the folded queue: drain at the rate in force, then the new window's rate
+            const uint32_t cap = n.cap_eff[x];
+            const bool on = n.online[x] != 0;
+            int64_t b = queued;
+            if (on) {
+                const int64_t done = int64_t(uint64_t(cap) * dt_ms / 1000u);
+                b = b > done ? b - done : 0;
+            }
+            if (db || on) n.backlog[x] = b;
+            const uint32_t cap_now = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, now_ms);
+            n.cap_eff[x] = cap_now;
+            refresh_gate(n, x, on, cap_now, b, credit_now);
+        } else {
+            if (db) n.backlog[x] = queued;
+            if (db || finalize) refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], queued, credit_now);
+        }
     }
     if (finalize) {
         // block sum of the committed credit, one atomic per block; the block that finishes a replica
@@ -216,8 +235,16 @@ void launch_fold(const Net& n, int finalize, const LaunchCtx& c)
 {
     const bool majority = finalize && (n.flags & 32u);
     if (majority) { Timed t(c, kFold); launch_kernel(c, k_count_online, peer_grid(n), 256, n); }
-    { Timed t(c, kFold); launch_kernel(c, k_fold, peer_grid(n), 256, n, finalize); }
+    { Timed t(c, kFold); launch_kernel(c, k_fold<false>, peer_grid(n), 256, n, finalize, 0u, 0u); }
     if (majority) { Timed t(c, kFold); launch_kernel(c, k_clear_online_count, (n.Rp + 127) / 128, 128, n); }
+}
+
+// The fold of the previous step and the time advance of this one in a single launch (not with
+// majority validation, whose online count needs a kernel of its own before the fold).
+void launch_fold_advance(const Net& n, int finalize, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c)
+{
+    Timed t(c, kFold);
+    launch_kernel(c, k_fold<true>, peer_grid(n), 256, n, finalize, dt_ms, now_ms);
 }
 
 void launch_rederive(const Net& n, const LaunchCtx& c)

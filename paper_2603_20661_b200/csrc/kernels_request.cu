@@ -285,6 +285,44 @@ void launch_fifo(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& 
     { Timed t(c, kFifo); launch_kernel(c, k_fifo_latency, dim3((count + 255) / 256, n.Rp), 256, n, first, count); }
 }
 
+// ---- batches to and from mapped host buffers ---------------------------------------------------------
+// One thread per request, consecutive threads on consecutive requests: every warp reads or writes whole
+// contiguous segments of the host buffers, so the bus carries full lines in request order.
+__global__ void __launch_bounds__(256) k_host_batch_in(Net n, HostBatch h, uint64_t first, uint32_t count)
+{
+    grid_dependency_enter();
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= count) return;
+    const size_t x = size_t(blockIdx.y) * n.Q + first + idx;
+    const_cast<uint32_t*>(n.origin)[x] = h.origin[x];
+    const_cast<uint16_t*>(n.len_in)[x] = h.len_in[x];
+    const_cast<uint16_t*>(n.len_out)[x] = h.len_out[x];
+}
+
+__global__ void __launch_bounds__(256) k_host_batch_out(Net n, HostBatch h, uint64_t first, uint32_t count)
+{
+    grid_dependency_enter();
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= count) return;
+    const size_t x = size_t(blockIdx.y) * n.Q + first + idx;
+    h.exec_a[x] = n.exec_a[x];
+    h.exec_b[x] = n.exec_b[x];
+    reinterpret_cast<int4*>(h.judges)[x] = reinterpret_cast<const int4*>(n.judges)[x];
+    h.outcome[x] = n.outcome[x];
+    h.rflags[x] = n.rflags[x];
+}
+
+void launch_host_batch_in(const Net& n, const HostBatch& h, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    Timed t(c, kHostBatch);
+    launch_kernel(c, k_host_batch_in, dim3((count + 255) / 256, n.Rp), 256, n, h, first, count);
+}
+void launch_host_batch_out(const Net& n, const HostBatch& h, uint64_t first, uint32_t count, const LaunchCtx& c)
+{
+    Timed t(c, kHostBatch);
+    launch_kernel(c, k_host_batch_out, dim3((count + 255) / 256, n.Rp), 256, n, h, first, count);
+}
+
 static dim3 warp_grid(const Net& n, uint32_t count) { return dim3((count + kWarpsPerBlock - 1) / kWarpsPerBlock, n.Rp); }
 
 void launch_dispatch(const Net& n, uint64_t first, uint32_t count, const LaunchCtx& c)

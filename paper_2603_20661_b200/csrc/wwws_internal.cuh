@@ -8,7 +8,7 @@ namespace wwws {
 
 // Kernel classes, for launch counts and optional event timing.
 enum KernelId : int { kPeerInit, kViewInit, kAdvance, kFold, kRederive, kCreditTotal, kGossipPeer,
-                      kGossipMerge, kGossipFixup, kGossipLists, kFifo, kDispatch, kDuel, kSettle, kStepFused, kKernelCount };
+                      kGossipMerge, kGossipFixup, kGossipLists, kFifo, kDispatch, kDuel, kSettle, kStepFused, kHostBatch, kKernelCount };
 
 // When enabled, every launch is bracketed by two events on the launching stream; read()
 // synchronises and returns the summed device time per kernel class.
@@ -56,9 +56,18 @@ inline void launch_kernel(const LaunchCtx& c, void (*kernel)(P...), dim3 grid, d
     cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
 }
 
+// Device-side addresses of a caller's mapped host buffers ([Rp][Q] like the bound arrays).
+struct HostBatch {
+    const uint32_t* origin; const uint16_t* len_in; const uint16_t* len_out;
+    int32_t* exec_a; int32_t* exec_b; int32_t* judges; uint8_t* outcome; uint8_t* rflags;
+};
+void launch_host_batch_in(const Net& n, const HostBatch& h, uint64_t first, uint32_t count, const LaunchCtx& c);
+void launch_host_batch_out(const Net& n, const HostBatch& h, uint64_t first, uint32_t count, const LaunchCtx& c);
+
 void launch_peer_init(const Net& n, const int64_t* credit0, const uint8_t* online0, uint32_t init_stale_max, const LaunchCtx& c);
 void launch_advance(const Net& n, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c);
 void launch_fold(const Net& n, int finalize, const LaunchCtx& c);
+void launch_fold_advance(const Net& n, int finalize, uint32_t dt_ms, uint32_t now_ms, const LaunchCtx& c);
 void launch_rederive(const Net& n, const LaunchCtx& c);
 void launch_credit_total(const Net& n, const LaunchCtx& c);
 void launch_gossip(const Net& n, uint32_t round, const LaunchCtx& c);

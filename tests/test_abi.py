@@ -81,5 +81,5 @@ def test_host_side_argument_checks():
     assert lib.wwws_gossip_round(None) == 1 and lib.wwws_dispatch_batch(None, 0, 1) == 1
     assert lib.wwws_gossip_round_static(None) == 1
     assert lib.wwws_destroy_network(None) == 0 and lib.wwws_kernel_launches(None) == 0
-    assert lib.wwws_profile_kernels() == 15
+    assert lib.wwws_profile_kernels() == 16
     assert lib.wwws_profile_kernel_name(7) == b"k_gossip_merge"
