@@ -75,8 +75,17 @@ def source_unchanged(rec):
 
 
 def find_counters(kernel, **match):
+    """The capture of `kernel` whose keys equal `match`; `workload` also matches a name listed in the
+    capture's `applies_to` (the same kernel at the same launch size on a network small enough to profile)."""
     for rec in read_counter_files():
-        if rec.get("kernel") == kernel and all(str(rec.get(k)) == str(v) for k, v in match.items()):
+        if rec.get("kernel") != kernel:
+            continue
+        ok = True
+        for k, v in match.items():
+            if k == "workload" and str(v) in rec.get("applies_to", "").replace(",", " ").split():
+                continue
+            ok = ok and str(rec.get(k)) == str(v)
+        if ok:
             return rec
     return None
 
@@ -156,7 +165,7 @@ REQUEST_KERNELS = ("k_advance", "k_step_fused", "k_fold", "k_fifo")
 class Leg:
     """One workload on this rank's GPU: the network, its step counter and the timed regions."""
 
-    def __init__(self, args, name, dev, world, rank, batch=None):
+    def __init__(self, args, name, dev, world, rank, batch=None, warmup=None):
         import torch
         from paper_2603_20661_b200 import synth
         from paper_2603_20661_b200.binding import Network
@@ -180,7 +189,7 @@ class Leg:
             self.net.set_option(4, args.host_io)
         if args.overlap is not None:
             self.net.set_option(3, args.overlap)
-        self.W, self.s = args.warmup, 0
+        self.W, self.s = (args.warmup if warmup is None else warmup), 0
         for _ in range(self.W):
             f, c, now, g = step_args(self.wl, self.s, self.W)
             self.net.step(f, c, now, g or self.s == 0); self.s += 1     # a gossip round in the warm-up whatever the phase
@@ -239,7 +248,7 @@ class Leg:
         return prof, {k: after[k] - before[k] for k in after}
 
 
-def rooflines(leg, prof, delta_b, sm_mhz):
+def rooflines(leg, prof, delta_b, sm_mhz, counters_workload=None):
     """HBM roofline of the gossip merge and of the request kernel, and the issue-slot roofline of
     the request kernel (warp instructions per request from the ncu capture on record)."""
     st, wl = leg.wl.settings, leg.wl
@@ -272,7 +281,7 @@ def rooflines(leg, prof, delta_b, sm_mhz):
         rate = per_launch / (req["ms_per_launch"] * 1e-3)
         req["requests_per_launch"] = per_launch
         req["requests_per_s"] = rate
-        rec = find_counters("k_step_fused", workload=leg.name)
+        rec = find_counters("k_step_fused", workload=counters_workload or leg.name)
         if rec and sm_mhz:
             ipr = float(rec["warp_instructions_per_request"])
             req["issue"] = {"bound": "alu", "warp_instr_per_request": ipr,
@@ -310,6 +319,26 @@ def run_compact_leg(args, name, dev, world, rank, sampler_index):
     return out
 
 
+SATURATED_BATCH = {"adversarial16k": 100000, "churn4k": 50000, "zipf1k": 10000}
+
+
+def run_saturated_leg(args, name, dev, world, rank, sampler_index):
+    """The request kernel alone on launches large enough to fill the GPU (the workload's whole request
+    stream of every replica in one step), on a fresh network so that the request mix is the workload's
+    own: the configurations' step sizes leave the kernel latency-bound, this is its throughput."""
+    leg = Leg(args, name, dev, world, rank, batch=SATURATED_BATCH[name], warmup=3)
+    sampler = ClockSampler(sampler_index).start() if rank == 0 else None
+    prof, delta_b = leg.profiled(3)
+    clocks = sampler.stop() if sampler else {"sm_mhz": None}
+    _, req, _ = rooflines(leg, prof, delta_b, clocks.get("sm_mhz"), counters_workload=name + "_saturated")
+    leg.close()
+    if req:
+        req["workload"] = name
+        req["batch_per_replica"] = SATURATED_BATCH[name]
+        req["offloaded_fraction"] = (delta_b["n_delegated"] + delta_b["n_fallback_local"] + delta_b["n_failed"]) / max(1, delta_b["n_requests"])
+    return req
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -344,18 +373,20 @@ def run_gpu(args):
 
     # ---- sustained: the same region repeated back to back for about a second of device time (each
     # repeat a whole number of gossip periods, so that all repeats hold the same work)
-    leg.align()
-    k_rep = K if K % wl.gossip_every == 0 else K * wl.gossip_every
-    reps = int(min(400, max(3, np.ceil(args.sustain_s * 1e3 / max(ms * k_rep / K, 1e-3)))))
-    sampler = ClockSampler(local).start() if rank == 0 else None
-    ms_rep, _ = leg.timed(k_rep, repeats=reps)
-    clocks_sustained = sampler.stop() if sampler else None
-    per_step = [m / k_rep for m in ms_rep]
-    sustained = {"repeats": len(ms_rep), "steps_per_repeat": k_rep, "device_seconds": sum(ms_rep) * 1e-3,
-                 "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
-                 "ms_per_step_max": max(per_step),
-                 "value_at_median": Rp * wl.batch * world / (statistics.median(per_step) * 1e-3),
-                 "clocks": clocks_sustained}
+    sustained, clocks_sustained = None, None
+    if args.sustain_s > 0:
+        leg.align()
+        k_rep = K if K % wl.gossip_every == 0 else K * wl.gossip_every
+        reps = int(min(400, max(3, np.ceil(args.sustain_s * 1e3 / max(ms * k_rep / K, 1e-3)))))
+        sampler = ClockSampler(local).start() if rank == 0 else None
+        ms_rep, _ = leg.timed(k_rep, repeats=reps)
+        clocks_sustained = sampler.stop() if sampler else None
+        per_step = [m / k_rep for m in ms_rep]
+        sustained = {"repeats": len(ms_rep), "steps_per_repeat": k_rep, "device_seconds": sum(ms_rep) * 1e-3,
+                     "ms_per_step_median": statistics.median(per_step), "ms_per_step_min": min(per_step),
+                     "ms_per_step_max": max(per_step),
+                     "value_at_median": Rp * wl.batch * world / (statistics.median(per_step) * 1e-3),
+                     "clocks": clocks_sustained}
 
     # ---- region B: K steps with per-kernel events (rooflines of the dominant kernel and of the request path)
     leg.align()
@@ -435,8 +466,10 @@ def run_gpu(args):
     # ---- the other large configurations, compactly (default run only) ---------------------------
     if args.legs and args.workload == DEFAULT_WORKLOAD and not args.batch:
         legs = [run_compact_leg(args, name, dev, world, rank, local) for name in EXTRA_LEGS]
+        sat = run_saturated_leg(args, args.workload, dev, world, rank, local)
         if line is not None:
             line["other_workloads"] = legs
+            line["roofline_request_path_saturated"] = sat
     if world > 1:
         dist.destroy_process_group()
     return line
@@ -535,7 +568,7 @@ def main(argv=None):
     ap.add_argument("--stream-run", type=int, default=0, help="requests per warp of the streaming kernel (WWWS_OPT_STREAM_RUN)")
     ap.add_argument("--host-io", type=int, default=0, help="wwws_step_host path: 0 by batch size, 1 mapped direct, 2 staged (WWWS_OPT_HOST_IO)")
     ap.add_argument("--overlap", type=int, default=None, help="mask of launches that may overlap their predecessor (WWWS_OPT_LAUNCH_OVERLAP)")
-    ap.add_argument("--sustain-s", type=float, default=1.0, help="device seconds of the repeated timed region")
+    ap.add_argument("--sustain-s", type=float, default=1.0, help="device seconds of the repeated timed region (0 skips it)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-legs", dest="legs", action="store_false", help="skip the compact legs on the other large workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing legs")

@@ -32,7 +32,7 @@ __device__ __forceinline__ uint64_t shfl64(unsigned mask, uint64_t v, int src)
 
 // Scores this lane's candidates of the window (o, blk); returns the lane-ascending fp32 sum of all
 // 32 scores (the same order of additions as a single thread would use) when `want_sum`.
-template <int L>
+template <int L, bool LOAD>
 __device__ __forceinline__ float score_lanes(const Net& n, Lanes<L>& w, uint32_t r, uint32_t o, uint32_t blk, bool want_sum)
 {
     constexpr int CP = Lanes<L>::CP;
@@ -49,8 +49,10 @@ __device__ __forceinline__ float score_lanes(const Net& n, Lanes<L>& w, uint32_t
 #pragma unroll
     for (int j = 0; j < CP; ++j) {
         const uint32_t id = kWin * blk + c0 + j;
-        const float wl = id < n.N ? wled[id] : 0.0f;
-        w.mine += candidate_weight(n, o, id, e[j], wl, w.sc[j]);          // sc = 0 when the weight is 0
+        float sc = candidate_score<LOAD>(n, uint32_t(e[j]), uint32_t(e[j] >> 32), wled[id]);   // padding columns: entry 0, weight 0
+        if (id == o) sc = 0.0f;                                            // the origin is not a candidate of its own request
+        w.sc[j] = sc;
+        w.mine += weight_q(sc);
     }
     float ssum = 0.0f;
     if (want_sum) {
@@ -89,7 +91,7 @@ __device__ __forceinline__ int draw_lanes(const Net& n, Lanes<L>& w, uint32_t q,
         int at = 32;
 #pragma unroll
         for (int j = 0; j < CP; ++j) {
-            const uint64_t x = weight_of(w.sc[j]);
+            const uint64_t x = weight_q(w.sc[j]);
             if (x > m) { m2 = m; m = x; at = int(w.sub) * CP + j; }
             else if (x > m2) m2 = x;
         }
@@ -119,7 +121,7 @@ __device__ __forceinline__ int draw_lanes(const Net& n, Lanes<L>& w, uint32_t q,
             uint64_t wp = 0;
 #pragma unroll
             for (int j = 0; j < CP; ++j) {
-                const uint64_t x = weight_of(w.sc[j]);
+                const uint64_t x = weight_q(w.sc[j]);
                 if (local < 0) {
                     if (r64 < lo + x) { local = j; wp = x; }
                     else lo += x;
@@ -141,7 +143,7 @@ __device__ __forceinline__ int draw_lanes(const Net& n, Lanes<L>& w, uint32_t q,
     return pick;
 }
 
-template <int L>
+template <int L, bool LOAD>
 __global__ void __launch_bounds__(128) k_step_lanes(Net n, uint64_t first, uint32_t count)
 {
     grid_dependency_enter();
@@ -169,10 +171,10 @@ __global__ void __launch_bounds__(128) k_step_lanes(Net n, uint64_t first, uint3
         int jd[4] = { -1, -1, -1, -1 };
         uint32_t oc = 0, blk = 0;
         float sa = 0.0f, ssum = 0.0f;
-        if (origin_offloads(n, r, o, rx, a)) {
+        if (origin_gate(n, r, o, rx, a)) {
             const int local_code = a;
             blk = pick_block(n, o, rx.w[2]);
-            ssum = score_lanes<L>(n, w, r, o, blk, n.score_sum != nullptr);
+            ssum = score_lanes<L, LOAD>(n, w, r, o, blk, n.score_sum != nullptr);
             // D5, D6: draw and probe until a peer accepts; for a duel go on with the challenger and the judges
             const bool duel = ppm(rx.w[1]) < n.p_duel;
             int found = -1, nj = 0, stage = 0;         // stage 0: executor, 1: challenger, 2: judges
@@ -185,7 +187,7 @@ __global__ void __launch_bounds__(128) k_step_lanes(Net n, uint64_t first, uint3
                 const int id = int(kWin * blk + pick);
                 if (stage < 2) {
                     w.n_probes++;
-                    if (probe_peer(n, r, rg, q, blk, pick)) {
+                    if (probe_gate(n, r, rg, q, blk, pick)) {
                         if (stage == 0) {
                             a = id;
                             if (!duel) break;
@@ -244,8 +246,14 @@ int step_lanes_for(uint64_t total)
 void launch_step_lanes(const Net& n, uint64_t first, uint32_t count, int lanes, const LaunchCtx& c)
 {
     Timed t(c, kStepFused);
-    if (lanes == 8) launch_kernel(c, k_step_lanes<8>, dim3((count + 15) / 16, n.Rp), 128, n, first, count);
-    else launch_kernel(c, k_step_lanes<4>, dim3((count + 31) / 32, n.Rp), 128, n, first, count);
+    const bool load = (n.flags & 2u) != 0;
+    if (lanes == 8) {
+        if (load) launch_kernel(c, k_step_lanes<8, true>, dim3((count + 15) / 16, n.Rp), 128, n, first, count);
+        else launch_kernel(c, k_step_lanes<8, false>, dim3((count + 15) / 16, n.Rp), 128, n, first, count);
+    } else {
+        if (load) launch_kernel(c, k_step_lanes<4, true>, dim3((count + 31) / 32, n.Rp), 128, n, first, count);
+        else launch_kernel(c, k_step_lanes<4, false>, dim3((count + 31) / 32, n.Rp), 128, n, first, count);
+    }
 }
 
 }  // namespace wwws

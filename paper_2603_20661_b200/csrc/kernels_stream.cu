@@ -27,7 +27,10 @@
 
 namespace wwws {
 
-constexpr uint32_t kSlots = 64;        // scored windows a warp holds at a time (draw + vote queues)
+#ifndef WWWS_STREAM_SLOTS
+#define WWWS_STREAM_SLOTS 64
+#endif
+constexpr uint32_t kSlots = WWWS_STREAM_SLOTS;   // scored windows a warp holds at a time (draw + vote queues), 33..64
 constexpr uint32_t kQ = 64;            // capacity of the score and finish queues
 
 // meta word of a slot: draws used (8) | probes used (8) | stage (2) | judges found (3) | near-boundary (1)
@@ -115,33 +118,6 @@ __device__ __forceinline__ void phase_origin(const Net& n, WarpPool& p, Warp& w)
 }
 
 // ---- score: D4 ------------------------------------------------------------------------------------
-// fp32 score of one candidate (0 when it is not eligible or its integer weight truncates to 0),
-// branch-free.  Same IEEE operations, in the same order, as candidate_weight().  Eligibility by
-// the entry is one range test on its bits 20..39 (advertised capacity and offline bit): capacity
-// in 1..2^19-1 and offline bit clear  <=>  (bits - 1) < 2^19 - 1; an entry that was never heard
-// of (0) and a padding column have capacity 0.  A ledger weight is never negative, so a score of
-// at least 2^-8 (integer weight >= 1) implies a positive weight.  The origin itself is taken out
-// of its own window by the caller.
-template <bool LOAD>
-__device__ __forceinline__ float candidate_score(const Net& n, uint32_t elo, uint32_t ehi, float wl)
-{
-    const uint32_t t = __funnelshift_r(elo, ehi, 20);
-    float spare = 1.0f;
-    if (LOAD) {
-        const float utilf = __fdiv_rn(__uint2float_rn((elo & kQMax) << 4), __fmul_rn(__uint2float_rn(t & kCapMax), n.uwf));
-        spare = fmaxf(__fsub_rn(1.0f, utilf), 0.0f);                 // capacity 0 gives inf or NaN here, and 0 after the max
-    }
-    const float sc = __fmul_rn(wl, spare);
-    const bool ok = ((t & 0xfffffu) - 1u) < kCapMax && sc >= 0.00390625f;
-    return ok ? sc : 0.0f;
-}
-
-// The integer weight of a stored score: trunc(256 sc), at most 2^56 (the same value as weight_of()).
-__device__ __forceinline__ unsigned long long weight_q(float sc)
-{
-    return __float2ull_rz(fminf(__fmul_rn(sc, 256.0f), 72057594037927936.0f));
-}
-
 template <bool SCORES, bool LOAD>
 __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, uint32_t m)
 {
@@ -188,7 +164,7 @@ __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, 
         }
         p.ident[slot] = e.x; p.where[slot] = e.y; p.meta[slot] = 0u; p.picks[slot] = 0u;
         if (SCORES && n.score_sum) n.score_sum[w.xbase + e.x] = ssum;
-        p.q_draw[(w.dr_head + w.dr_n + w.lane) & (kSlots - 1)] = uint8_t(slot);
+        p.q_draw[(w.dr_head + w.dr_n + w.lane) % kSlots] = uint8_t(slot);
     }
     w.sc_head += m; w.sc_n -= m; w.n_free -= m; w.dr_n += m;
 }
@@ -204,7 +180,7 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
     uint32_t slot = 0;
     uint4 fin = make_uint4(0, 0, 0, 0);
     if (active) {
-        slot = p.q_draw[(w.dr_head + w.lane) & (kSlots - 1)];
+        slot = p.q_draw[(w.dr_head + w.lane) % kSlots];
         if (!index_ok(n, slot, kSlots, 501)) slot = 0;
         const uint32_t meta = p.meta[slot], where = p.where[slot], idx = p.ident[slot];
         uint32_t picks = p.picks[slot];
@@ -300,8 +276,8 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
     __syncwarp();                               // every lane has read its queue entry: the ring's head may be reused by the pushes below
     const uint32_t mc = __ballot_sync(kFull, kind == kCont), mv = __ballot_sync(kFull, kind == kVote), mf = __ballot_sync(kFull, to_fin);
     w.dr_head += m; w.dr_n -= m;
-    if (kind == kCont) p.q_draw[(w.dr_head + w.dr_n + __popc(mc & w.lt)) & (kSlots - 1)] = uint8_t(slot);
-    if (kind == kVote) p.q_vote[(w.vo_head + w.vo_n + __popc(mv & w.lt)) & (kSlots - 1)] = uint8_t(slot);
+    if (kind == kCont) p.q_draw[(w.dr_head + w.dr_n + __popc(mc & w.lt)) % kSlots] = uint8_t(slot);
+    if (kind == kVote) p.q_vote[(w.vo_head + w.vo_n + __popc(mv & w.lt)) % kSlots] = uint8_t(slot);
     if (to_fin) {
         p.q_fin[(w.fi_head + w.fi_n + __popc(mf & w.lt)) & (kQ - 1)] = fin;
         p.free_slots[w.n_free + __popc(mf & w.lt)] = uint8_t(slot);
@@ -314,7 +290,7 @@ __device__ __forceinline__ void phase_vote(const Net& n, WarpPool& p, Warp& w, u
 {
     const bool active = w.lane < m;
     if (active) {
-        uint32_t slot = p.q_vote[(w.vo_head + w.lane) & (kSlots - 1)];
+        uint32_t slot = p.q_vote[(w.vo_head + w.lane) % kSlots];
         if (!index_ok(n, slot, kSlots, 504)) slot = 0;
         const uint32_t meta = p.meta[slot], where = p.where[slot], idx = p.ident[slot], picks = p.picks[slot];
         const uint32_t blk = (where >> 16) & 0x7ffu, o = where & 0xffffu, q = uint32_t(w.first + idx);
@@ -368,7 +344,7 @@ __device__ __forceinline__ void phase_finish(const Net& n, WarpPool& p, Warp& w,
 enum : int { phOrigin, phScore, phDraw, phVote, phFinish, phDone };
 
 template <bool GREEDY, bool SCORES, bool LOAD>
-__global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, uint32_t count)
+__global__ void __launch_bounds__(32, kSlots > 48 ? 16 : kSlots > 40 ? 19 : 22) k_step_stream(Net n, uint64_t first, uint32_t count)
 {
     grid_dependency_enter();
     __shared__ WarpPool p;
@@ -380,7 +356,8 @@ __global__ void __launch_bounds__(32, 16) k_step_stream(Net n, uint64_t first, u
     w.chunk = blockIdx.x; w.stride = gridDim.x;
     w.sc_head = w.sc_n = w.dr_head = w.dr_n = w.vo_head = w.vo_n = w.fi_head = w.fi_n = 0;
     w.n_free = kSlots;
-    p.free_slots[w.lane] = uint8_t(w.lane); p.free_slots[w.lane + 32] = uint8_t(w.lane + 32);
+    p.free_slots[w.lane] = uint8_t(w.lane);
+    if (w.lane + 32u < kSlots) p.free_slots[w.lane + 32] = uint8_t(w.lane + 32);
     WideAcc acc;
 #pragma unroll
     for (int k = 0; k <= int(sSloMet); ++k) acc.c[k] = 0;

@@ -71,6 +71,55 @@ __device__ __forceinline__ uint64_t candidate_weight(const Net& n, uint32_t o, u
     return W;
 }
 
+// fp32 score of one candidate (0 when it is not eligible or its integer weight truncates to 0),
+// branch-free.  Same IEEE operations, in the same order, as candidate_weight().  Eligibility by
+// the entry is one range test on its bits 20..39 (advertised capacity and offline bit): capacity
+// in 1..2^19-1 and offline bit clear  <=>  (bits - 1) < 2^19 - 1; an entry that was never heard
+// of (0) and a padding column have capacity 0.  A ledger weight is never negative, so a score of
+// at least 2^-8 (integer weight >= 1) implies a positive weight.  The origin itself is taken out
+// of its own window by the caller.
+template <bool LOAD>
+__device__ __forceinline__ float candidate_score(const Net& n, uint32_t elo, uint32_t ehi, float wl)
+{
+    const uint32_t t = __funnelshift_r(elo, ehi, 20);
+    float spare = 1.0f;
+    if (LOAD) {
+        const float utilf = __fdiv_rn(__uint2float_rn((elo & kQMax) << 4), __fmul_rn(__uint2float_rn(t & kCapMax), n.uwf));
+        spare = fmaxf(__fsub_rn(1.0f, utilf), 0.0f);                 // capacity 0 gives inf or NaN here, and 0 after the max
+    }
+    const float sc = __fmul_rn(wl, spare);
+    const bool ok = ((t & 0xfffffu) - 1u) < kCapMax && sc >= 0.00390625f;
+    return ok ? sc : 0.0f;
+}
+
+// The integer weight of a stored score: trunc(256 sc), at most 2^56 (the same value as weight_of()).
+__device__ __forceinline__ unsigned long long weight_q(float sc)
+{
+    return __float2ull_rz(fminf(__fmul_rn(sc, 256.0f), 72057594037927936.0f));
+}
+
+// D1, D2 from the origin's gate word (see refresh_gate): true if the request goes to the network,
+// else `code` is the local / dropped / failed code.  Same decisions as origin_offloads().
+__device__ __forceinline__ bool origin_gate(const Net& n, uint32_t r, uint32_t o, const Rnd4& rx, int& code)
+{
+    code = -3;
+    if (o >= n.N) { set_error(n, eArg, o); return false; }
+    const uint32_t g = reinterpret_cast<const uint32_t*>(n.gate)[2 * (size_t(r) * n.N + o) + 1];
+    if (!(g & kGateOnline)) return false;
+    code = (g & kGateNoCap) ? -4 : -1;
+    return ppm(rx.w[0]) < (g & kGateFreq);
+}
+
+// D6 from the drawn candidate's gate word: one load and the probe's random word.
+__device__ __forceinline__ bool probe_gate(const Net& n, uint32_t r, uint32_t rg, uint32_t q, uint32_t blk, int pick)
+{
+    if (!index_ok(n, kWin * blk + uint32_t(pick), n.N, 410)) return false;
+    const uint32_t thr = reinterpret_cast<const uint32_t*>(n.gate)[2 * (size_t(r) * n.N + kWin * blk + pick)];
+    const Rnd4 y = draw(n, q, uint32_t(pick) >> 2, rg, kProbe);
+    const uint32_t sel = uint32_t(pick) & 3u;
+    return ppm(sel == 0 ? y.w[0] : sel == 1 ? y.w[1] : sel == 2 ? y.w[2] : y.w[3]) < thr;
+}
+
 // The integer weight that candidate_weight() derives from a score.
 __device__ __forceinline__ uint64_t weight_of(float sc)
 {

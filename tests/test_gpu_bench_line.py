@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("workload,extra", [("tiers64", []), ("zipf1k", ["--replicas", "8"])])
 def test_bench_prints_one_complete_json_line(workload, extra):
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", workload, "--steps", "4", "--warmup", "3",
-                          "--no-cpu-all-cores"] + extra, capture_output=True, text=True, timeout=600, cwd=ROOT)
+                          "--no-cpu-all-cores", "--sustain-s", "0.05"] + extra, capture_output=True, text=True, timeout=600, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
     lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
     assert len(lines) == 1
@@ -35,3 +35,8 @@ def test_bench_prints_one_complete_json_line(workload, extra):
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    # the K-step region repeated back to back, and the request path's line with the stated target beside it
+    su = d["sustained"]
+    assert su["repeats"] >= 3 and su["ms_per_step_min"] <= su["ms_per_step_median"] <= su["ms_per_step_max"]
+    rq = d["roofline_request_path"]
+    assert rq["target_frac"] == 0.6 and rq["target_met"] == (rq["frac"] >= 0.6) and rq["requests_per_s"] > 0
