@@ -70,3 +70,22 @@ def test_launcher_command_and_missing_devices():
         out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--workload", "tiny"],
                              capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
         assert out.returncode != 0 and "--gpus 2" in out.stderr and out.stdout.strip() == ""
+
+
+def test_counter_files_on_record_are_found_and_tied_to_their_source():
+    """The ncu counters bench.py quotes (DRAM traffic of the merge, warp instructions per request of
+    the request kernels) come from small text files written when a capture is taken; each names the
+    kernel's source file and its digest, and a figure is withheld once the source has changed."""
+    sys.path.insert(0, ROOT)
+    import bench
+    recs = bench.read_counter_files()
+    assert len(recs) >= 4 and all({"kernel", "commit", "source", "source_sha256", "command"} <= set(r) for r in recs)
+    merge = bench.find_counters("k_gossip_merge", n_peers=16384, fanout_k=4, flags=3)
+    assert merge and 4.29e9 < float(merge["dram_bytes_per_replica_round"]) < 4.5e9       # compulsory 2 * 8 * N^2 = 4.295e9
+    for wl in ("adversarial16k", "zipf1k", "zipf1k_saturated", "adversarial16k_saturated"):
+        rec = bench.find_counters("k_step_fused", workload=wl)
+        assert rec and 50 < float(rec["warp_instructions_per_request"]) < 1000, wl
+        assert 1 <= float(rec["active_lanes_per_instruction"]) <= 32
+    assert bench.find_counters("k_step_fused", workload="no_such_workload") is None
+    assert bench.source_unchanged(merge) in (True, False)
+    assert bench.source_unchanged({"source": "bench.py", "source_sha256": "0" * 64}) is False
