@@ -390,12 +390,14 @@ def run_gpu(args):
 
     # ---- region B: K steps with per-kernel events (rooflines of the dominant kernel and of the request path)
     leg.align()
+    sampler = ClockSampler(local).start() if rank == 0 else None
     prof, delta_b = leg.profiled(K)
+    clocks_profiled = sampler.stop() if sampler else None
     peak, peak_kind = measured_peaks()
     total_ms = sum(v[0] for v in prof.values())
     dom = max(prof, key=lambda k: prof[k][0])
     kernels = {k: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_ms} for k, v in prof.items()}
-    sm_mhz = (clocks_sustained or {}).get("sm_mhz") or (clocks or {}).get("sm_mhz")
+    sm_mhz = (clocks_profiled or {}).get("sm_mhz") or (clocks or {}).get("sm_mhz")     # the clock while these kernels were timed
     roof_merge, roof_req, t_req = rooflines(leg, prof, delta_b, sm_mhz)
     roofline = roof_merge if dom == "k_gossip_merge" else roof_req
     # the whole timed region A against HBM: algorithmic bytes of its gossip rounds and requests over its duration

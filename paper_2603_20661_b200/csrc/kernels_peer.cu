@@ -114,23 +114,34 @@ __global__ void k_fold(Net n, int finalize_requested, uint32_t dt_ms, uint32_t n
     long long csum = 0;
     if (j < n.N) {
         const size_t x = size_t(r) * n.N + j;
+        // Most peers are untouched by a batch (16,000 requests on 262,144 peers): every table is
+        // read, but written only where its value changes.
         const long long db = n.d_backlog[x];
-        const int64_t queued = n.backlog[x] + db;
+        const int64_t queued_before = n.backlog[x], queued = queued_before + db;
         if (db) n.d_backlog[x] = 0;
         int64_t credit_now = n.credit[x];
+        bool ledger_changed = false;
         if (n.flags & 16u) {
             n.in_deg[x] = 0;                         // per-peer item counts of the batch's queueing pass
             n.blk_spent[x] = finalize ? 0 : n.blk_spent[x] + n.d_spent[x];
             n.d_spent[x] = 0;
         }
         if (finalize) {
-            const int64_t c = n.credit[x] + n.d_credit[x];
-            const uint32_t w = n.wins[x] + n.d_wins[x], d = n.duels[x] + n.d_duels[x];
-            n.credit[x] = c; n.wins[x] = w; n.duels[x] = d;
-            n.d_credit[x] = 0; n.d_wins[x] = 0; n.d_duels[x] = 0;
-            const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
-            n.stake[x] = st;
-            n.w_led[size_t(r) * n.ld + j] = ledger_weight(n, st, w, d);
+            const long long dc = n.d_credit[x];
+            const uint32_t dw = n.d_wins[x], dd = n.d_duels[x];
+            const int64_t c = credit_now + dc;
+            if (dc) { n.credit[x] = c; n.d_credit[x] = 0; }
+            if (dw | dd) {
+                const uint32_t w = n.wins[x] + dw, d = n.duels[x] + dd;
+                if (dw) { n.wins[x] = w; n.d_wins[x] = 0; }
+                if (dd) { n.duels[x] = d; n.d_duels[x] = 0; }
+            }
+            if (dc || dw || dd) {                    // stake and ledger weight are functions of (credit, wins, duels)
+                const int64_t st = (c > 0 ? c : 0) * int64_t(n.stake_pm[x]) / 1000;
+                n.stake[x] = st;
+                n.w_led[size_t(r) * n.ld + j] = ledger_weight(n, st, n.wins[x], n.duels[x]);
+                ledger_changed = true;
+            }
             csum = c;
             credit_now = c;
         }
@@ -143,13 +154,13 @@ __global__ void k_fold(Net n, int finalize_requested, uint32_t dt_ms, uint32_t n
                 const int64_t done = int64_t(uint64_t(cap) * dt_ms / 1000u);
                 b = b > done ? b - done : 0;
             }
-            if (db || on) n.backlog[x] = b;
+            if (b != queued_before) n.backlog[x] = b;
             const uint32_t cap_now = cap_eff_at(n, n.cap_true[x], n.prio_flag[x] != 0, j, r + n.replica_offset, now_ms);
-            n.cap_eff[x] = cap_now;
-            refresh_gate(n, x, on, cap_now, b, credit_now);
+            if (cap_now != cap) n.cap_eff[x] = cap_now;
+            if (b != queued_before || cap_now != cap || ledger_changed) refresh_gate(n, x, on, cap_now, b, credit_now);
         } else {
             if (db) n.backlog[x] = queued;
-            if (db || finalize) refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], queued, credit_now);
+            if (db || ledger_changed) refresh_gate(n, x, n.online[x] != 0, n.cap_eff[x], queued, credit_now);
         }
     }
     if (finalize) {
