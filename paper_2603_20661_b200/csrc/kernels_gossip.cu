@@ -31,13 +31,19 @@ __global__ void k_gossip_peer(Net n, uint32_t round)
         uint32_t open = (1u << n.fanout_k) - 1u;     // slots still looking for a partner
         for (uint32_t a = 0; a < n.gossip_tries && open; ++a) {
             const Rnd4 g = draw(n, i, round, rg, kGossip + 256u * a);
+            // the candidates of all open slots first, their entries fetched together (one memory round
+            // trip per attempt instead of one per slot), then the decisions
+            uint32_t cand[4];
+            uint64_t ent[4];
 #pragma unroll
             for (uint32_t s = 0; s < 4; ++s) {
-                if (!(open >> s & 1u)) continue;
-                const uint32_t p = below(g.w[s], n.N);
-                if (p == i) continue;
-                const uint64_t e = row[p];
-                if (e != 0 && !(e & kOffBit) && index_ok(n, p, n.N, 101)) { part[s] = int32_t(p); open &= ~(1u << s); }
+                cand[s] = below(g.w[s], n.N);
+                ent[s] = (open >> s & 1u) ? row[cand[s]] : 0ull;
+            }
+#pragma unroll
+            for (uint32_t s = 0; s < 4; ++s) {
+                if (!(open >> s & 1u) || cand[s] == i) continue;
+                if (ent[s] != 0 && !(ent[s] & kOffBit) && index_ok(n, cand[s], n.N, 101)) { part[s] = int32_t(cand[s]); open &= ~(1u << s); }
             }
         }
     }

@@ -58,6 +58,38 @@ def test_one_replica_of_the_full_run_matches_the_oracle(name, replica, steps):
     g.close()
 
 
+@pytest.mark.parametrize("name,batch,replica", [("zipf1k", 10000, 131), ("adversarial16k", 100000, 9)])
+def test_one_replica_of_the_saturated_launch_matches_the_oracle(name, batch, replica):
+    """The benchmark's saturated leg: a replica's whole request stream in one step (2.56 M and 1.6 M
+    requests per launch; every warp of the streaming kernel runs through hundreds of requests).
+    One replica is checked completely against the oracle run on that replica alone."""
+    from paper_2603_20661_b200.binding import Network
+    wl = synth.make_workload(name)
+    wl.batch = batch
+    g = Network(wl.settings, wl.peers, wl.batch)
+    g.bind_requests(wl.requests, scores=False)
+    one = synth.slice_replicas(wl, replica, replica + 1)
+    one.batch = batch
+    o = Oracle(one.settings, one.peers)
+    o.bind_requests(one.requests)
+    steps = min(2, wl.n_steps)
+    for s in range(steps):
+        args = (s * batch, batch, wl.step_now_ms(s), s == 0)
+        g.step(*args)
+        o.run_step(*args)
+    upto = steps * batch
+    rg, ro = g.results(), o.results()
+    for k in ("exec_a", "exec_b", "judges", "outcome", "flags"):
+        assert np.array_equal(rg[k][replica, :upto], ro[k][0, :upto]), f"{name}: {k} differs"
+    for t in TABLE_NAMES:
+        assert np.array_equal(g.table(t)[replica].astype(np.int64), o.table(t)[0]), f"{name}: table {t} differs"
+    assert np.array_equal(g.stats()[replica], o.stats()[0]), f"{name}: counters differ"
+    sd = g.stats()
+    assert np.all(sd[:-1, 0] == upto)
+    assert np.array_equal(sd[:-1, 17].astype(np.int64), wl.peers["credit0"].sum(axis=1))
+    g.close()
+
+
 @pytest.mark.skipif(os.environ.get("WWWS_MAX_SIZE") != "1",
                     reason="the oracle needs over a minute and about 100 GB of host memory at 65,535 peers: set WWWS_MAX_SIZE=1")
 @pytest.mark.parametrize("n_peers", [32768, 65535])
