@@ -232,15 +232,14 @@ __global__ void __launch_bounds__(128) k_step_lanes(Net n, uint64_t first, uint3
 }
 
 // Lanes per request for a launch of `total` requests over all replicas, or 0 when the launch is
-// large enough for the thread-per-request kernel: the sub-warp kernel pays only while all its
-// threads are resident at once (about 100,000 threads at its register count).  Measured on 148 SMs:
-// 16,000 requests 39 us (one thread) / 31 us (4 lanes) / 32 us (8 lanes); 4,000 requests 38 / 28 / 23 us;
-// 500 requests 30 / 22 / 20 us.
+// large enough for the streaming kernel.  Measured on 148 SMs (4,096-peer network, 1,000 requests per
+// replica), 8 lanes / 4 lanes / streaming: 2,000 requests 20.9 / 24.0 / 25.1 us; 8,000: 23.0 / 26.1 /
+// 25.4; 12,000: 24.4 / 27.1 / 26.8; 16,000: 30.6 / 27.5 / 27.1; 24,000: 36.0 / 29.1 / 27.8;
+// 32,000: 41.5 / 38.7 / 29.1.  Four lanes per request are never the fastest any more and remain as
+// an implementation that can be forced (WWWS_OPT_STEP_KERNEL).
 int step_lanes_for(uint64_t total)
 {
-    if (total <= 8192) return 8;
-    if (total <= 25000) return 4;
-    return 0;
+    return total <= 12288 ? 8 : 0;
 }
 
 void launch_step_lanes(const Net& n, uint64_t first, uint32_t count, int lanes, const LaunchCtx& c)

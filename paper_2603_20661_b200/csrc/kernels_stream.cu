@@ -176,6 +176,11 @@ template <bool GREEDY, bool SCORES>
 __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, uint32_t m)
 {
     const bool active = w.lane < m;
+    // A full batch takes every request one draw further and regroups.  A partial batch means the warp
+    // has nothing else to fill its lanes with (its input is exhausted, or its windows are all taken):
+    // then each lane takes its request on, draw after draw, until it leaves the draw phase - fewer
+    // rounds at the end of a run, which is what a launch that gives a warp only a chunk or two is made of.
+    const bool run_on = m < 32u;
     int kind = kIdle;
     uint32_t slot = 0;
     uint4 fin = make_uint4(0, 0, 0, 0);
@@ -188,82 +193,87 @@ __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, u
         bool near = (meta >> 21) & 1u;
         const uint32_t blk = (where >> 16) & 0x7ffu, q = uint32_t(w.first + idx);
         const size_t cbase = w.pbase + kWin * blk;
-        const unsigned long long G0 = p.G[0][slot], G1 = p.G[1][slot], G2 = p.G[2][slot], G3 = p.G[3][slot];
-        const unsigned long long S = G0 + G1 + G2 + G3;
-        int pick = -1;
-        if (S != 0) {
-            const uint32_t k = n_draws++;
-            uint32_t g;
-            unsigned long long wp;
-            if (GREEDY) {
-                // greedy rule: highest weight, lowest candidate on ties; flagged when the runner-up is within 1e-5
-                unsigned long long m1 = 0, m2 = 0;
+        unsigned long long G0 = p.G[0][slot], G1 = p.G[1][slot], G2 = p.G[2][slot], G3 = p.G[3][slot];
+#pragma unroll 1
+        for (;;) {
+            const unsigned long long S = G0 + G1 + G2 + G3;
+            int pick = -1;
+            if (S != 0) {
+                const uint32_t k = n_draws++;
+                uint32_t g;
+                unsigned long long wp;
+                if (GREEDY) {
+                    // greedy rule: highest weight, lowest candidate on ties; flagged when the runner-up is within 1e-5
+                    unsigned long long m1 = 0, m2 = 0;
 #pragma unroll 4
-                for (int c = 0; c < int(kWin); ++c) {
-                    const unsigned long long x = weight_q(p.S[c][slot]);
-                    if (x > m1) { m2 = m1; m1 = x; pick = c; }
-                    else if (x > m2) m2 = x;
-                }
-                if (m2 != 0 && m1 - m2 <= m1 / 100000ull) near = true;
-                g = uint32_t(pick) >> 3; wp = m1;
-            } else {
-                unsigned long long u;
-                if (k & 1u) u = p.ycache[slot];
-                else {
-                    const Rnd4 y = draw(n, q, k >> 1, w.rg, kDraw);
-                    u = (unsigned long long)y.w[0] << 32 | y.w[1];
-                    p.ycache[slot] = (unsigned long long)y.w[2] << 32 | y.w[3];
-                }
-                const unsigned long long r64 = __umul64hi(u, S);
-                // the group whose interval holds r64, then the candidate inside it, without branches:
-                // the pick is the number of inclusive prefix sums that do not exceed r64
-                const unsigned long long c1 = G0 + G1, c2 = c1 + G2;
-                g = uint32_t(r64 >= G0) + uint32_t(r64 >= c1) + uint32_t(r64 >= c2);
-                unsigned long long lo = g == 0 ? 0ull : g == 1 ? G0 : g == 2 ? c1 : c2, acc = lo;
-                uint32_t cnt = 0;
-                wp = 0;
+                    for (int c = 0; c < int(kWin); ++c) {
+                        const unsigned long long x = weight_q(p.S[c][slot]);
+                        if (x > m1) { m2 = m1; m1 = x; pick = c; }
+                        else if (x > m2) m2 = x;
+                    }
+                    if (m2 != 0 && m1 - m2 <= m1 / 100000ull) near = true;
+                    g = uint32_t(pick) >> 3; wp = m1;
+                } else {
+                    unsigned long long u;
+                    if (k & 1u) u = p.ycache[slot];
+                    else {
+                        const Rnd4 y = draw(n, q, k >> 1, w.rg, kDraw);
+                        u = (unsigned long long)y.w[0] << 32 | y.w[1];
+                        p.ycache[slot] = (unsigned long long)y.w[2] << 32 | y.w[3];
+                    }
+                    const unsigned long long r64 = __umul64hi(u, S);
+                    // the group whose interval holds r64, then the candidate inside it, without branches:
+                    // the pick is the number of inclusive prefix sums that do not exceed r64
+                    const unsigned long long c1 = G0 + G1, c2 = c1 + G2;
+                    g = uint32_t(r64 >= G0) + uint32_t(r64 >= c1) + uint32_t(r64 >= c2);
+                    unsigned long long lo = g == 0 ? 0ull : g == 1 ? G0 : g == 2 ? c1 : c2, acc = lo;
+                    uint32_t cnt = 0;
+                    wp = 0;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const unsigned long long x = weight_q(p.S[8 * g + j][slot]);
-                    const bool below = acc + x <= r64;                   // candidate j ends at or before r64
-                    if (!below && cnt == uint32_t(j)) wp = x;            // the first one that does not is the pick
-                    acc += x;
-                    if (below) { lo = acc; ++cnt; }
+                    for (int j = 0; j < 8; ++j) {
+                        const unsigned long long x = weight_q(p.S[8 * g + j][slot]);
+                        const bool below = acc + x <= r64;                   // candidate j ends at or before r64
+                        if (!below && cnt == uint32_t(j)) wp = x;            // the first one that does not is the pick
+                        acc += x;
+                        if (below) { lo = acc; ++cnt; }
+                    }
+                    pick = int(8u * g + cnt);
+                    const unsigned long long d1 = r64 - lo, d2 = lo + wp - 1 - r64;
+                    if ((d1 < d2 ? d1 : d2) <= S / 100000ull) near = true;
+                    if (cnt >= 8u) pick = -1;                                // cannot happen: the group sums are the sums of the weights in play
                 }
-                pick = int(8u * g + cnt);
-                const unsigned long long d1 = r64 - lo, d2 = lo + wp - 1 - r64;
-                if ((d1 < d2 ? d1 : d2) <= S / 100000ull) near = true;
-                if (cnt >= 8u) pick = -1;                                // cannot happen: the group sums are the sums of the weights in play
+                if (pick >= 0) {
+                    if (SCORES && stage == 0 && n.score_a) fin.x = __float_as_uint(p.S[pick][slot]);     // the executor's score, if this pick accepts
+                    p.S[pick][slot] = 0.0f;
+                    if (g == 0) G0 -= wp; else if (g == 1) G1 -= wp; else if (g == 2) G2 -= wp; else G3 -= wp;
+                }
             }
-            if (pick >= 0) {
-                if (SCORES && stage == 0 && n.score_a) fin.x = __float_as_uint(p.S[pick][slot]);     // the executor's score, if this pick accepts
-                p.S[pick][slot] = 0.0f;
-                p.G[g][slot] = (g == 0 ? G0 : g == 1 ? G1 : g == 2 ? G2 : G3) - wp;
+            if (pick >= 0 && !index_ok(n, kWin * blk + uint32_t(pick), n.N, 502)) pick = -1;
+            kind = kCont;
+            if (pick < 0) kind = stage == 0 ? kFinNone : (stage == 2 && nj ? kVote : kFinCancel);
+            else if (stage < 2) {
+                ++n_probes;
+                // D6: the drawn candidate answers by its true state and its own accept policy (its gate)
+                const uint32_t thr = reinterpret_cast<const uint32_t*>(n.gate)[2 * (cbase + pick)];
+                const Rnd4 y = draw(n, q, uint32_t(pick) >> 2, w.rg, kProbe);
+                const uint32_t sel = uint32_t(pick) & 3u;
+                const bool accepted = ppm(sel == 0 ? y.w[0] : sel == 1 ? y.w[1] : sel == 2 ? y.w[2] : y.w[3]) < thr;
+                if (accepted) {
+                    if (stage == 0) {
+                        picks = uint32_t(pick);
+                        if (SCORES && n.score_a) n.score_a[w.xbase + idx] = __uint_as_float(fin.x);
+                        if (where & kWhereDuel) { stage = 1; if (n_probes >= n.max_probes) kind = kFinCancel; }
+                        else kind = kFinPlain;
+                    } else { picks |= uint32_t(pick) << 5; stage = 2; }
+                } else if (n_probes >= n.max_probes) kind = stage == 0 ? kFinNone : kFinCancel;
+            } else {
+                if (n.online[cbase + pick]) { picks |= uint32_t(pick) << (10u + 5u * nj); ++nj; }
+                if (nj >= n.n_judges) kind = kVote;
             }
-        }
-        if (pick >= 0 && !index_ok(n, kWin * blk + uint32_t(pick), n.N, 502)) pick = -1;
-        kind = kCont;
-        if (pick < 0) kind = stage == 0 ? kFinNone : (stage == 2 && nj ? kVote : kFinCancel);
-        else if (stage < 2) {
-            ++n_probes;
-            // D6: the drawn candidate answers by its true state and its own accept policy (its gate)
-            const uint32_t thr = reinterpret_cast<const uint32_t*>(n.gate)[2 * (cbase + pick)];
-            const Rnd4 y = draw(n, q, uint32_t(pick) >> 2, w.rg, kProbe);
-            const uint32_t sel = uint32_t(pick) & 3u;
-            const bool accepted = ppm(sel == 0 ? y.w[0] : sel == 1 ? y.w[1] : sel == 2 ? y.w[2] : y.w[3]) < thr;
-            if (accepted) {
-                if (stage == 0) {
-                    picks = uint32_t(pick);
-                    if (SCORES && n.score_a) n.score_a[w.xbase + idx] = __uint_as_float(fin.x);
-                    if (where & kWhereDuel) { stage = 1; if (n_probes >= n.max_probes) kind = kFinCancel; }
-                    else kind = kFinPlain;
-                } else { picks |= uint32_t(pick) << 5; stage = 2; }
-            } else if (n_probes >= n.max_probes) kind = stage == 0 ? kFinNone : kFinCancel;
-        } else {
-            if (n.online[cbase + pick]) { picks |= uint32_t(pick) << (10u + 5u * nj); ++nj; }
-            if (nj >= n.n_judges) kind = kVote;
+            if (!(run_on && kind == kCont)) break;
         }
         if (kind == kCont || kind == kVote) {
+            p.G[0][slot] = G0; p.G[1][slot] = G1; p.G[2][slot] = G2; p.G[3][slot] = G3;
             p.meta[slot] = n_draws | n_probes << 8 | stage << 16 | nj << 18 | (near ? 1u << 21 : 0u);
             p.picks[slot] = picks;
         } else {

@@ -311,7 +311,7 @@ def test_random_configurations_match_oracle(seed):
     rng = np.random.default_rng(1000 + seed)
     N = int(rng.choice([2, 3, 9, 31, 32, 33, 64, 97, 200, 513]))
     Rp = int(rng.integers(1, 4))
-    B = int(rng.choice([1, 7, 60, 120, 3500, 9000]))       # the large ones reach the 4-lane and the one-thread step kernels
+    B = int(rng.choice([1, 7, 60, 120, 3500, 9000]))       # the large ones reach the streaming step kernel when the kernel is chosen by launch size
     Q = max(360, 3 * B)
     n_blk = (N + 31) // 32
     kw = dict(fanout_k=int(rng.integers(1, 5)), gossip_tries=int(rng.integers(1, 9)), max_probes=int(rng.integers(1, 8)),
