@@ -176,11 +176,11 @@ template <bool GREEDY, bool SCORES>
 __device__ __forceinline__ void phase_draw(const Net& n, WarpPool& p, Warp& w, uint32_t m)
 {
     const bool active = w.lane < m;
-    // A full batch takes every request one draw further and regroups.  A partial batch means the warp
-    // has nothing else to fill its lanes with (its input is exhausted, or its windows are all taken):
-    // then each lane takes its request on, draw after draw, until it leaves the draw phase - fewer
-    // rounds at the end of a run, which is what a launch that gives a warp only a chunk or two is made of.
-    const bool run_on = m < 32u;
+    // A batch normally takes every request one draw further and regroups.  Once the warp's input is
+    // exhausted a partial batch has nothing left to fill its lanes with: then each lane takes its
+    // request on, draw after draw, until it leaves the draw phase - fewer rounds at the end of a run,
+    // which is what a launch that gives a warp only a chunk or two is made of.
+    const bool run_on = m < 32u && w.chunk >= w.n_chunks;
     int kind = kIdle;
     uint32_t slot = 0;
     uint4 fin = make_uint4(0, 0, 0, 0);
