@@ -132,29 +132,25 @@ __device__ __forceinline__ void phase_score(const Net& n, WarpPool& p, Warp& w, 
         const uint32_t self = (o >> 5) == blk ? (o & 31u) : 32u;
         float ssum = 0.0f;
 #pragma unroll 1
-        for (int h = 0; h < 2; ++h) {                                  // 16 candidates at a time: four 32-byte loads in flight
-            E4 v[4];
-            float4 f[4];
+        for (int g = 0; g < 4; ++g) {                                  // one 8-candidate group at a time: two 32-byte loads in flight
+            E4 v[2];
+            float4 f[2];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v[i] = ld_entries(row + 128 * h + 32 * i);
+            for (int i = 0; i < 2; ++i) v[i] = ld_entries(row + 64 * g + 32 * i);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) f[i] = __ldg(wl4 + 4 * h + i);
+            for (int i = 0; i < 2; ++i) f[i] = __ldg(wl4 + 2 * g + i);
+            unsigned long long gsum = 0;
 #pragma unroll
-            for (int g2 = 0; g2 < 2; ++g2) {
-                unsigned long long gsum = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int k = 8 * g2 + j;
-                    const uint32_t c = 16u * h + k;
-                    const float wl = (k & 3) == 0 ? f[k >> 2].x : (k & 3) == 1 ? f[k >> 2].y : (k & 3) == 2 ? f[k >> 2].z : f[k >> 2].w;
-                    float sc = candidate_score<LOAD>(n, v[k >> 2].lo[k & 3], v[k >> 2].hi[k & 3], wl);
-                    if (SCORES) sc = self != c ? sc : 0.0f;            // the checked sum leaves the origin out as it goes
-                    p.S[c][slot] = sc;
-                    gsum += weight_q(sc);
-                    if (SCORES) ssum = __fadd_rn(ssum, sc);
-                }
-                p.G[2 * h + g2][slot] = gsum;
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t c = 8u * g + k;
+                const float wl = (k & 3) == 0 ? f[k >> 2].x : (k & 3) == 1 ? f[k >> 2].y : (k & 3) == 2 ? f[k >> 2].z : f[k >> 2].w;
+                float sc = candidate_score<LOAD>(n, v[k >> 2].lo[k & 3], v[k >> 2].hi[k & 3], wl);
+                if (SCORES) sc = self != c ? sc : 0.0f;            // the checked sum leaves the origin out as it goes
+                p.S[c][slot] = sc;
+                gsum += weight_q(sc);
+                if (SCORES) ssum = __fadd_rn(ssum, sc);
             }
+            p.G[g][slot] = gsum;
         }
         if (!SCORES && self < 32u) {
             // the origin is not a candidate of its own request: take it out of its window
