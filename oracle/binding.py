@@ -58,7 +58,9 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        # WWWS_ORACLE_LIBRARY: another build of the oracle (the pin tests load deliberately broken copies
+        # through it to show that each planted mistake is caught)
+        L = C.CDLL(os.environ.get("WWWS_ORACLE_LIBRARY") or build())
         L.orc_create.restype = C.c_void_p
         L.orc_create.argtypes = [C.POINTER(_Config), C.POINTER(_PeerInit)]
         L.orc_destroy.argtypes = [C.c_void_p]

@@ -37,6 +37,12 @@
  *                      recomputed peer by peer and window by window from the second Philox,
  *                      plus hand cases and the active-window frequency
  *
+ *   all of the above   tests/test_oracle_mutations.py plants some fifty single mistakes (a dropped
+ *                      term, a wrong sign or constant, an off-by-one, swapped operands) in copies of
+ *                      this file and requires the pins to fail on each; the three that survived its
+ *                      first run (advertised queue units, judges must be online, hop latency) got
+ *                      pins of their own
+ *
  * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
  */
 #include <stdint.h>

@@ -362,3 +362,43 @@ def test_in_block_validation_counts_uncovered_payments():
     o3 = Oracle(st, pa); o3.bind_requests(rq)
     o3.dispatch_batch(0, 6); o3.duel_judge(); o3.settle_credits(True)
     assert o3.stats_dict()["n_uncovered"] == 0
+
+
+def test_judges_are_peers_that_are_truly_online():
+    """J2: a drawn candidate serves as a judge only if it is online now, whatever the origin's view
+    still believes; executor and challenger must be online too (the probe reaches the real peer)."""
+    N = 10
+    st, pa, rq = make_net(N, n_requests=600, seed=4, p_duel_ppm=1_000_000, n_judges=3, max_probes=8,
+                          peers=requester_first(N, credit0=10 ** 7))
+    o = Oracle(st, pa); o.bind_requests(rq)
+    gone = (3, 6, 7)
+    for j in gone:
+        o.poke_peer(0, j, online=0)                      # crashed since the last gossip round: the views do not know yet
+    assert np.all(np.array([(int(o.view()[0, 0, j]) >> 39) & 1 for j in gone]) == 0)
+    o.dispatch_batch(0, 600); o.duel_judge(); o.settle_credits(True)
+    res = o.results()
+    decided = np.isin(res["outcome"][0], (1, 2, 3))
+    assert decided.sum() > 300
+    jd = res["judges"][0][decided]
+    assert not np.isin(jd, gone).any() and not np.isin(res["exec_a"][0], gone).any() and not np.isin(res["exec_b"][0], gone).any()
+    assert np.all((jd >= 0).sum(axis=1) == 3)            # six peers remain online besides A and B: always three judges
+    # every online peer other than the requester does serve as a judge at some point
+    assert set(np.unique(jd[jd >= 0])) == set(range(1, N)) - set(gone)
+
+
+def test_hop_latency_is_added_to_delegated_requests_only():
+    """S4: a delegated request pays the network hop once, a locally served one does not."""
+    def total_latency(hop):
+        st, pa, rq = make_net(3, n_requests=40, origin=np.array([1, 0] * 20), lens=(600, 400), p_duel_ppm=0, hop_ms=hop,
+                              peers={"offload_ppm": np.array([1_000_000, 0, 0]), "cap_true_tok_s": np.array([1000, 2000, 4000])})
+        o = Oracle(st, pa); o.bind_requests(rq)
+        o.dispatch_batch(0, 40); o.duel_judge(); o.settle_credits(True)
+        ex = o.results()["exec_a"][0]
+        return o.stats_dict()["sum_latency_ms"], int((ex >= 0).sum()), int((ex == -1).sum()), o.stats_dict()["slo_met"]
+    lat0, deleg0, local0, met0 = total_latency(0)
+    lat7, deleg7, local7, met7 = total_latency(37)
+    assert (deleg0, local0) == (deleg7, local7) == (20, 20)
+    assert lat7 - lat0 == 37 * deleg0
+    # with a hop longer than any deadline no delegated request meets it, the local ones are unaffected
+    _, _, _, met_far = total_latency(10_000)
+    assert met0 > met_far and met_far <= local0

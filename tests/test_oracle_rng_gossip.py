@@ -250,3 +250,30 @@ def test_partner_choice_is_uniform_and_slots_are_independent():
     exp = np.array([m * 1, m * (m - 1) * 3, m * (m - 1) * (m - 2)], float) / m ** 3
     ok, s2, _ = chi2_ok(np.bincount(distinct, minlength=4)[1:], distinct.size * exp)
     assert ok, s2
+
+
+def test_own_entry_advertises_capacity_and_queue_in_16_token_units():
+    """G1: an online peer's fresh entry carries its version, its advertised capacity (true rate x
+    misreport factor, saturating at 2^19 - 1) and its queue in 16-token units (saturating at
+    2^20 - 1); the views of the peers that pull it take the same entry."""
+    from tests.helpers import entry_cap, entry_q
+    N = 12
+    cap = np.arange(N) * 700 + 100
+    st, pa, _ = make_net(N, fanout_k=3, seed=2, peers={"cap_true_tok_s": cap, "misreport_mul": np.where(np.arange(N) % 4 == 0, 4, 1)})
+    o = Oracle(st, pa)
+    queues = {1: 15, 2: 16, 3: 1000, 4: 123_457, 5: (1 << 24) + 5, 6: 1 << 40}
+    for j, b in queues.items():
+        o.poke_peer(0, j, backlog=b)
+    o.gossip_round()
+    v = o.view()[0]
+    ver = o.table("ver")[0]
+    for j in range(N):
+        own = v[j, j]
+        assert int(entry_ver(own)) == ver[j] and int(entry_offline(own)) == 0
+        assert int(entry_cap(own)) == min((1 << 19) - 1, int(cap[j]) * (4 if j % 4 == 0 else 1))
+        assert int(entry_q(own)) == min((1 << 20) - 1, queues.get(j, 0) >> 4)
+    # whoever holds the current version of j holds exactly that entry
+    for i in range(N):
+        for j in range(N):
+            if int(entry_ver(v[i, j])) == ver[j]:
+                assert (int(v[i, j]) | OFFBIT) == (int(v[j, j]) | OFFBIT)
